@@ -1,0 +1,169 @@
+/*
+ * fastav.h -- C ABI of the B200-native FastAV prune step.
+ *
+ * FastAV (Section 2.2 of the paper) prunes the token sequence of an audio-visual LLM during
+ * prefill: at a pruning layer it scores every token by the attention the last query token(s)
+ * pay to it (Eq. 4:  s = mean_h softmax(Q_last K^T)),  removes the lowest-scoring P% and lets
+ * the following layers run on the survivors only.  The same step serves the "global" stage at
+ * the middle layer and the "fine" stage at every later layer.  This library is that step:
+ *
+ *     fastav_score    Eq. 4, generalised to R scored rows, grouped-query heads, varlen batches
+ *     fastav_select   "tokens with the lowest P% scores are removed": top-k keep set
+ *     fastav_compact  the survivor layout: gather hidden states, position ids, K and V rows
+ *     fastav_prune    all three in one enqueue
+ *
+ * Conventions shared by every call
+ *   - Plain C.  No CUDA types: `stream` is a cudaStream_t passed as void*.
+ *   - Every data pointer is a DEVICE pointer unless its comment says "host".  The params struct
+ *     is read on the host at call time.
+ *   - The caller owns every buffer (inputs, outputs, workspace).  The library allocates nothing
+ *     and keeps no state between calls.
+ *   - Calls only enqueue work on `stream` and return; they never synchronise.  On a negative
+ *     return value nothing was enqueued.
+ *   - bf16 tensors are token-major.  Strides are in elements; the innermost dimension
+ *     (head_dim, hidden) is contiguous.  Rows must start on 16-byte boundaries.
+ *   - A batch is a packed ("varlen") concatenation of sequences: sequence b owns tokens
+ *     [cu_seqlens[b], cu_seqlens[b+1]) and scored rows [cu_qlens[b], cu_qlens[b+1]).
+ *   - Conditions only the device can see (a keep count outside [0, n_b], more protected tokens
+ *     than k_b) are handled by clamping and reported by OR-ing FASTAV_DEV_* bits into
+ *     *device_status (optional, may be NULL; the caller zeroes it).  Nothing traps.
+ */
+#ifndef FASTAV_H_
+#define FASTAV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FASTAV_VERSION 100 /* major*10000 + minor*100 + patch */
+
+/* return codes */
+#define FASTAV_OK 0
+#define FASTAV_ERR_INVALID_ARG (-1) /* NULL required pointer, batch < 1, Hq % Hkv != 0, stride < row, counts inconsistent, in/out overlap */
+#define FASTAV_ERR_UNSUPPORTED (-2) /* head_dim not 64/128, hidden % 8 != 0, misaligned pointer or stride */
+#define FASTAV_ERR_WORKSPACE (-3)   /* workspace NULL, misaligned or smaller than fastav_workspace_bytes() */
+#define FASTAV_ERR_CUDA (-4)        /* a launch failed; fastav_last_cuda_error() has the runtime's text */
+#define FASTAV_ERR_TIMEOUT (-5)     /* reserved: every device-side wait is bounded */
+
+/* params.flags */
+#define FASTAV_CAUSAL 1u              /* scored row r sees keys j <= q_idx[r] only (the model's own mask) */
+#define FASTAV_PROTECT_QUERY_ROWS 2u  /* the scored rows' tokens always survive (and count toward k_b) */
+#define FASTAV_KEEP_IDX_GLOBAL 4u     /* keep_idx holds indices into the packed batch, not sequence-local ones */
+
+/* bits OR-ed into *device_status */
+#define FASTAV_DEV_K_CLAMPED 1        /* some keep_counts[b] was outside [0, n_b] and was clamped */
+#define FASTAV_DEV_PROTECT_OVERFLOW 2 /* more protected tokens than k_b: the lowest-index ones were kept */
+#define FASTAV_DEV_WAIT_EXPIRED 4     /* a bounded wait inside a kernel ran out; results of that call are invalid */
+#define FASTAV_DEV_BAD_INDEX 8        /* fastav_compact met a keep_idx entry outside its sequence and skipped that row */
+
+/*
+ * Shapes of one prune call (host memory).  The counts that fix grid sizes and output sizes are
+ * host scalars because the caller knows them without a device round trip: k_b is a function of
+ * n_b ("lowest P%" -> k_b = n_b - floor(P n_b)).
+ */
+typedef struct fastav_params {
+  int32_t batch;                    /* B >= 1 */
+  int32_t total_tokens, max_seqlen; /* N = cu_seqlens[B]; max_b n_b */
+  int32_t total_q, max_qlen;        /* sum_b R_b = cu_qlens[B]; max_b R_b */
+  int32_t total_keep, max_keep;     /* sum_b k_b; max_b k_b (upper bounds are fine) */
+  int32_t num_q_heads, num_kv_heads, head_dim; /* Hq % Hkv == 0; head_dim 64 or 128 */
+  int32_t hidden;                   /* D, a multiple of 8 */
+  int64_t q_stride_tok, q_stride_head;                                 /* q  [total_q, Hq, head_dim] */
+  int64_t k_stride_tok, k_stride_head, v_stride_tok, v_stride_head;     /* k,v [N, Hkv, head_dim]    */
+  int64_t ko_stride_tok, ko_stride_head, vo_stride_tok, vo_stride_head; /* outputs [total_keep, Hkv, head_dim] */
+  float softmax_scale;              /* <= 0 selects 1/sqrt(head_dim); 1.0 is Eq. 4 as printed */
+  uint32_t flags;                   /* FASTAV_CAUSAL | FASTAV_PROTECT_QUERY_ROWS | FASTAV_KEEP_IDX_GLOBAL */
+} fastav_params;
+
+/* Library version (FASTAV_VERSION of the build). */
+int32_t fastav_version(void);
+
+/* Static text for a return code. */
+const char* fastav_status_string(int32_t status);
+
+/* Text of the last CUDA runtime error seen by this thread inside the library ("" if none). */
+const char* fastav_last_cuda_error(void);
+
+/*
+ * Bytes of device workspace that fastav_score / fastav_select / fastav_prune need for these
+ * shapes (out_bytes: host).  The workspace must be 256-byte aligned; its contents are scratch
+ * and need no initialisation.  Two calls running concurrently need two workspaces.
+ */
+int32_t fastav_workspace_bytes(const fastav_params* params, size_t* out_bytes);
+
+/*
+ * Importance scores, Eq. 4 (Section 2.2, "Fine pruning"), without forming the L x L map.
+ * For sequence b, token j:
+ *
+ *   scores_out[cu_seqlens[b] + j] =
+ *       1/(Hq R_b) * sum_{r < R_b} sum_{h < Hq} softmax_{j' in V(r)}( scale <q[r,h,:], k[j', h/G, :]> )[j]
+ *
+ * with G = Hq/Hkv, V(r) = all keys of the sequence, or {j' <= q_idx[r]} under FASTAV_CAUSAL
+ * (keys outside V(r) get 0 from that row).  R_b = 1 at the last token is Eq. 4 itself.
+ *
+ *   q          [total_q, Hq, head_dim] bf16  query vectors of the scored rows (as the layer's
+ *                                            attention uses them, i.e. after RoPE)
+ *   q_idx      [total_q] int32               sequence-local token index of each scored row
+ *   cu_qlens   [B+1] int32
+ *   k          [N, Hkv, head_dim] bf16
+ *   cu_seqlens [B+1] int32
+ *   lse_opt    reserved, pass NULL
+ *   scores_out [N] fp32 (written for every token; a sequence with R_b = 0 gets zeros)
+ */
+int32_t fastav_score(const fastav_params* params, const void* q, const int32_t* q_idx, const int32_t* cu_qlens,
+                     const void* k, const int32_t* cu_seqlens, const float* lse_opt, float* scores_out,
+                     void* workspace, size_t workspace_bytes, int32_t* device_status, void* stream);
+
+/*
+ * "Tokens with the lowest P% scores are removed" (Section 2.2): per sequence keep the
+ * keep_counts[b] highest-scoring tokens; equal scores go to the lower index; protected tokens
+ * (protect_opt[j] != 0, and the scored rows' tokens under FASTAV_PROTECT_QUERY_ROWS) rank above
+ * every score.  Survivors are written in ascending index order.
+ *
+ *   scores       [N] fp32 (finite)
+ *   keep_counts  [B] int32          k_b; values outside [0, n_b] are clamped (FASTAV_DEV_K_CLAMPED)
+ *   protect_opt  [N] uint8 or NULL
+ *   q_idx, cu_qlens                 read only under FASTAV_PROTECT_QUERY_ROWS (else may be NULL)
+ *   keep_idx_out [total_keep] int32 sequence-local indices (packed-batch indices under
+ *                                   FASTAV_KEEP_IDX_GLOBAL), ascending within each sequence
+ *   cu_keep_out  [B+1] int32        prefix sums of the clamped k_b
+ */
+int32_t fastav_select(const fastav_params* params, const float* scores, const int32_t* cu_seqlens,
+                      const int32_t* keep_counts, const uint8_t* protect_opt, const int32_t* q_idx,
+                      const int32_t* cu_qlens, int32_t* keep_idx_out, int32_t* cu_keep_out, void* workspace,
+                      size_t workspace_bytes, int32_t* device_status, void* stream);
+
+/*
+ * Survivor layout (what "iteratively refining the token set" in Section 2.2 leaves for the next
+ * layer): output row cu_keep[b] + i is input row cu_seqlens[b] + keep_idx[cu_keep[b] + i] of
+ *
+ *   hidden  [N, hidden] bf16   -> hidden_out [total_keep, hidden]
+ *   pos     [N] int32          -> pos_out    [total_keep]      (position ids are carried, never renumbered)
+ *   k, v    [N, Hkv, head_dim] -> k_out, v_out [total_keep, Hkv, head_dim] (strides from params)
+ *
+ * Bit-exact copies.  Any in/out pair may be NULL (both NULL) and is skipped.  Outputs must not
+ * overlap inputs.  Needs no workspace.
+ */
+int32_t fastav_compact(const fastav_params* params, const int32_t* keep_idx, const int32_t* cu_keep,
+                       const int32_t* cu_seqlens, const void* hidden_in, void* hidden_out, const int32_t* pos_in,
+                       int32_t* pos_out, const void* k_in, void* k_out, const void* v_in, void* v_out,
+                       int32_t* device_status, void* stream);
+
+/*
+ * The whole prune step of one pruning layer (Fig. 3; Section 2.2): fastav_score, fastav_select
+ * and fastav_compact enqueued back to back.  scores_out, keep_idx_out and cu_keep_out are still
+ * written, so the caller can inspect or reuse them.  Arguments as in the three calls above.
+ */
+int32_t fastav_prune(const fastav_params* params, const void* q, const int32_t* q_idx, const int32_t* cu_qlens,
+                     const void* k, const void* v, const int32_t* cu_seqlens, const int32_t* keep_counts,
+                     const uint8_t* protect_opt, const void* hidden_in, const int32_t* pos_in, float* scores_out,
+                     int32_t* keep_idx_out, int32_t* cu_keep_out, void* hidden_out, int32_t* pos_out, void* k_out,
+                     void* v_out, void* workspace, size_t workspace_bytes, int32_t* device_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FASTAV_H_ */

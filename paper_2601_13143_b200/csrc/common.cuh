@@ -1,0 +1,60 @@
+// Internal declarations shared by the kernels and the C-ABI layer.  Nothing here is exported.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "fastav.h"
+
+namespace fastav {
+
+constexpr int kNumSMs = 148;          // B200: 2 dies x 74 SMs; grids are sized in multiples of this
+constexpr float kLog2e = 1.4426950408889634f;
+
+// Device-side view of one call's shapes (a trimmed fastav_params, passed by value).
+struct Shapes {
+  int batch, total_tokens, max_seqlen, total_q, max_qlen, total_keep, max_keep;
+  int hq, hkv, group, dim, hidden;
+  long long q_st, q_sh, k_st, k_sh, v_st, v_sh, ko_st, ko_sh, vo_st, vo_sh;
+  float scale_log2;  // softmax scale * log2(e): logits are kept in base-2 units
+  unsigned flags;
+};
+
+// Carved from the caller's workspace by plan_workspace(); all offsets 256-byte aligned.
+struct Workspace {
+  size_t total = 0;
+  // generic / narrow score
+  size_t stats_off = 0;     // float2 [total_q * Hq][stat_tiles]   per-tile (max, sum-exp2)
+  size_t lse_off = 0;       // float  [total_q * Hq]               log2-sum-exp2 per (row, head)
+  size_t partial_off = 0;   // float  [Hkv][N]                     per-KV-head score partials
+  size_t logits_off = 0;    // float  [Hq * R][N] (narrow path only; 0 bytes otherwise)
+  // select
+  size_t keys_off = 0;      // uint32 [N] (only when a sequence does not fit in shared memory)
+  int stat_tiles = 0;
+};
+
+Workspace plan_workspace(const fastav_params& p);
+
+// ---- launchers (each returns cudaGetLastError() after its launches) -------------------------
+cudaError_t launch_score(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
+                         const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
+                         unsigned char* ws, cudaStream_t stream);
+
+cudaError_t launch_score_generic(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
+                                 const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
+                                 unsigned char* ws, cudaStream_t stream);
+
+cudaError_t launch_select(const Shapes& s, const Workspace& w, const float* scores, const int32_t* cu_seqlens,
+                          const int32_t* keep_counts, const uint8_t* protect, const int32_t* q_idx,
+                          const int32_t* cu_qlens, int32_t* keep_idx, int32_t* cu_keep, unsigned char* ws,
+                          int32_t* device_status, cudaStream_t stream);
+
+cudaError_t launch_compact(const Shapes& s, const int32_t* keep_idx, const int32_t* cu_keep,
+                           const int32_t* cu_seqlens, const void* hidden_in, void* hidden_out, const int32_t* pos_in,
+                           int32_t* pos_out, const void* k_in, void* k_out, const void* v_in, void* v_out,
+                           int32_t* device_status, cudaStream_t stream);
+
+__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace fastav

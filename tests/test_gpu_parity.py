@@ -1,0 +1,313 @@
+"""GPU parity: every C-ABI entry point against the CPU oracle on the same seeded bits."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import parity
+from conftest import bf16_bits
+from paper_2601_13143_b200 import fastav
+from paper_2601_13143_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def _sync_status(buf):
+    torch.cuda.synchronize()
+    return int(buf.device_status.cpu())
+
+
+# ---- score ------------------------------------------------------------------------------------
+
+SCORE_CASES = [
+    # lens, rows, hq, hkv, d
+    ([1], [1], 4, 4, 64),
+    ([2], [1], 4, 1, 64),
+    ([7], [3], 8, 2, 64),
+    ([8, 9], [1, 4], 7, 1, 128),
+    ([127], [4], 28, 4, 128),
+    ([128, 129], [3, 1], 28, 4, 128),
+    ([1000], [64], 8, 2, 64),
+    ([333, 0, 65], [4, 0, 3], 32, 8, 128),
+    ([200], [0], 8, 2, 64),
+    ([2500], [5], 4, 2, 128),
+]
+
+
+@pytest.mark.parametrize("lens,rows,hq,hkv,d", SCORE_CASES)
+@pytest.mark.parametrize("causal", [True, False])
+def test_score_matches_oracle(lens, rows, hq, hkv, d, causal):
+    p = W.random_problem(seed=sum(lens) + hq, lens=lens, rows=rows, keeps=[n // 2 for n in lens], num_q_heads=hq,
+                         num_kv_heads=hkv, head_dim=d, hidden=64, duplicate_keys=3, trailing_rows=False)
+    p.causal = causal
+    buf = parity.to_device(p)
+    buf.scores.fill_(float("nan"))
+    buf.score()
+    torch.cuda.synchronize()
+    ref = parity.oracle_scores(p)
+    parity.assert_scores_close(buf.scores, ref, f"lens={lens} rows={rows}")
+    got = buf.scores.cpu().numpy()
+    cu = p.cu_seqlens.numpy()
+    for b, (n, r) in enumerate(zip(lens, rows)):
+        if n and min(r, n):
+            assert abs(got[cu[b]:cu[b + 1]].sum() - 1.0) < 1e-4
+    # bit-reproducible
+    first = buf.scores.clone()
+    buf.score()
+    torch.cuda.synchronize()
+    assert torch.equal(first.view(torch.int32), buf.scores.view(torch.int32))
+
+
+def test_score_softmax_scale_one_is_eq4_as_printed():
+    p = W.random_problem(seed=3, lens=[50], rows=[1], keeps=[25], num_q_heads=4, num_kv_heads=2, head_dim=64, hidden=64)
+    p.softmax_scale = 1.0
+    p.k = (p.k.float() * 0.25).to(torch.bfloat16)
+    buf = parity.to_device(p)
+    buf.score()
+    torch.cuda.synchronize()
+    parity.assert_scores_close(buf.scores, parity.oracle_scores(p), "scale 1")
+
+
+def test_score_strided_qkv_views():
+    """q and k as views into one packed [tokens, Hq + 2 Hkv, d] projection output."""
+    g = torch.Generator().manual_seed(21)
+    n, hq, hkv, d = 300, 8, 2, 64
+    packed = torch.randn(n, hq + 2 * hkv, d, generator=g).to(torch.bfloat16)
+    p = W.random_problem(seed=1, lens=[n], rows=[4], keeps=[100], num_q_heads=hq, num_kv_heads=hkv, head_dim=d, hidden=64)
+    dev = packed.cuda()
+    q_view, k_view, v_view = dev[n - 4:, :hq], dev[:, hq:hq + hkv], dev[:, hq + hkv:]
+    buf = fastav.make_buffers(q=q_view, q_idx=p.q_idx.cuda(), cu_qlens=p.cu_qlens.cuda(), k=k_view, v=v_view,
+                              cu_seqlens=p.cu_seqlens.cuda(), keep_counts=p.keep_counts.cuda(), hidden=p.hidden.cuda(),
+                              pos=p.pos.cuda(), softmax_scale=p.softmax_scale, flags=fastav.FASTAV_CAUSAL,
+                              lens=[n], rows=[4], keeps=[100])
+    buf.prune()
+    torch.cuda.synchronize()
+    bits = bf16_bits(packed)
+    ref = oracle.prune(bits[n - 4:, :hq], bits[:, hq:hq + hkv], bits[:, hq + hkv:], bf16_bits(p.hidden), p.pos.numpy(),
+                       p.cu_seqlens.numpy(), p.cu_qlens.numpy(), p.q_idx.numpy(), p.keep_counts.numpy(), p.softmax_scale,
+                       True, protect_rows=False)
+    parity.assert_scores_close(buf.scores, ref["scores"], "strided")
+    if np.array_equal(buf.keep_idx.cpu().numpy()[:100], ref["keep_idx"]):
+        parity.assert_bits_equal(buf.k_out, ref["k"], "k")
+        parity.assert_bits_equal(buf.v_out, ref["v"], "v")
+        parity.assert_bits_equal(buf.hidden_out, ref["hidden"], "hidden")
+
+
+# ---- select -----------------------------------------------------------------------------------
+
+def _select_case(lens, keeps, scores, protect=None, rows=None, q_idx=None, global_idx=False, protect_rows=False):
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    rows = [0] * len(lens) if rows is None else rows
+    cuq = np.concatenate([[0], np.cumsum(rows)]).astype(np.int32)
+    q_idx = np.zeros(0, dtype=np.int32) if q_idx is None else np.asarray(q_idx, dtype=np.int32)
+    clamped = [min(max(k, 0), n) for k, n in zip(keeps, lens)]
+    flags = (fastav.FASTAV_PROTECT_QUERY_ROWS if protect_rows else 0) | (fastav.FASTAV_KEEP_IDX_GLOBAL if global_idx else 0)
+    params = fastav.make_params(batch=len(lens), total_tokens=int(cu[-1]), max_seqlen=max(lens), total_q=int(cuq[-1]),
+                                max_qlen=max(rows), total_keep=sum(clamped), max_keep=max(clamped), num_q_heads=4,
+                                num_kv_heads=2, head_dim=64, hidden=64, flags=flags)
+    dev = lambda a, dt: torch.as_tensor(np.asarray(a), dtype=dt).cuda()
+    ws = torch.empty(max(fastav.fastav_workspace_bytes(params), 256), dtype=torch.uint8, device="cuda")
+    keep_idx = torch.full((max(sum(clamped), 1) + 8,), -7, dtype=torch.int32, device="cuda")
+    cu_keep = torch.full((len(lens) + 1,), -7, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    fastav.fastav_select(params, dev(scores, torch.float32), dev(cu, torch.int32), dev(keeps, torch.int32),
+                         None if protect is None else dev(protect, torch.uint8), dev(q_idx, torch.int32) if len(q_idx) else None,
+                         dev(cuq, torch.int32), keep_idx, cu_keep, ws, status)
+    torch.cuda.synchronize()
+    ref_idx, ref_cu = oracle.select(scores, cu, keeps, protect, protect_rows, q_idx, cuq, global_idx)
+    assert cu_keep.cpu().tolist() == ref_cu.tolist()
+    got = keep_idx.cpu().numpy()
+    assert got[:len(ref_idx)].tolist() == ref_idx.tolist()
+    assert (got[len(ref_idx):] == -7).all()          # nothing written past the end
+    return int(status.cpu())
+
+
+def test_select_matches_oracle_with_ties_protection_and_edge_sizes():
+    rng = np.random.default_rng(0)
+    lens = [1, 2, 7, 8, 9, 127, 128, 129, 1000, 0, 33, 1025, 4097]
+    keeps = [1, 1, 3, 8, 0, 64, 127, 129, 400, 0, 32, 1, 4096]
+    n = sum(lens)
+    scores = (rng.integers(0, 50, size=n) / 1024.0).astype(np.float32)          # heavy ties
+    assert _select_case(lens, keeps, scores) == 0
+    protect = (rng.random(n) < 0.05).astype(np.uint8)
+    assert _select_case(lens, keeps, scores, protect) & ~fastav.FASTAV_DEV_PROTECT_OVERFLOW == 0
+    assert _select_case(lens, keeps, scores, protect, global_idx=True) & ~fastav.FASTAV_DEV_PROTECT_OVERFLOW == 0
+    smooth = rng.random(n).astype(np.float32) * 1e-3
+    assert _select_case(lens, keeps, smooth) == 0
+
+
+def test_select_general_floats_negative_zero_and_inf():
+    scores = np.array([0.0, -0.0, 1.5, -2.0, np.inf, 3e-39, -3e-39, 1.5, -np.inf, 0.0], dtype=np.float32)
+    for k in range(0, 11):
+        _select_case([10], [min(k, 10)], scores)
+
+
+def test_select_clamps_and_reports():
+    scores = np.linspace(0, 1, 20).astype(np.float32)
+    status = _select_case([10, 10], [12, -3], scores)
+    assert status & fastav.FASTAV_DEV_K_CLAMPED
+    protect = np.zeros(20, dtype=np.uint8)
+    protect[[1, 3, 5, 7]] = 1
+    status = _select_case([10, 10], [2, 5], scores, protect)
+    assert status & fastav.FASTAV_DEV_PROTECT_OVERFLOW
+
+
+def test_select_protects_query_rows():
+    rng = np.random.default_rng(4)
+    lens, rows = [40, 50], [3, 2]
+    scores = rng.random(90).astype(np.float32)
+    scores[[37, 38, 39, 40 + 48, 40 + 49]] = 0.0          # the scored rows would otherwise be dropped first
+    assert _select_case(lens, [10, 10], scores, rows=rows, q_idx=[37, 38, 39, 48, 49], protect_rows=True) == 0
+
+
+def test_select_sequence_longer_than_shared_memory():
+    rng = np.random.default_rng(5)
+    n = 70_000
+    scores = (rng.integers(0, 5000, size=n) / 65536.0).astype(np.float32)
+    assert _select_case([n, 100], [n // 3, 50], scores=np.concatenate([scores, rng.random(100).astype(np.float32)])) == 0
+
+
+# ---- compact ----------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("hkv,d,hid", [(2, 64, 64), (4, 128, 3584), (8, 128, 4096), (1, 64, 8)])
+def test_compact_matches_oracle(hkv, d, hid):
+    rng = np.random.default_rng(hkv * 100 + d)
+    lens = [37, 0, 129, 1]
+    keeps = [10, 0, 129, 1]
+    p = W.random_problem(seed=hid, lens=lens, rows=[1, 0, 1, 1], keeps=keeps, num_q_heads=hkv * 2, num_kv_heads=hkv,
+                         head_dim=d, hidden=hid)
+    cu = p.cu_seqlens.numpy()
+    keep_idx = np.concatenate([np.sort(rng.choice(n, size=k, replace=False)) for n, k in zip(lens, keeps)]).astype(np.int32)
+    cu_keep = np.concatenate([[0], np.cumsum(keeps)]).astype(np.int32)
+    ref = oracle.compact(keep_idx, cu_keep, cu, bf16_bits(p.hidden), p.pos.numpy(), bf16_bits(p.k), bf16_bits(p.v))
+    buf = parity.to_device(p, flags=0)
+    for t in (buf.hidden_out, buf.k_out, buf.v_out):
+        t.view(torch.int16).fill_(0x7FC1)
+    buf.pos_out.fill_(-1)
+    buf.keep_idx[:len(keep_idx)].copy_(torch.as_tensor(keep_idx))
+    buf.cu_keep.copy_(torch.as_tensor(cu_keep))
+    buf.compact()
+    assert _sync_status(buf) == 0
+    for name in ("hidden", "pos", "k", "v"):
+        parity.assert_bits_equal(getattr(buf, name + "_out"), ref[name], name)
+    # global indices, only the K pair
+    buf.params.flags = fastav.FASTAV_KEEP_IDX_GLOBAL
+    global_idx = np.concatenate([cu[b] + keep_idx[cu_keep[b]:cu_keep[b + 1]] for b in range(len(lens))]).astype(np.int32)
+    buf.keep_idx[:len(global_idx)].copy_(torch.as_tensor(global_idx))
+    buf.k_out.zero_()
+    fastav.fastav_compact(buf.params, buf.keep_idx, buf.cu_keep, buf.cu_seqlens, k_in=buf.k, k_out=buf.k_out)
+    torch.cuda.synchronize()
+    parity.assert_bits_equal(buf.k_out, ref["k"], "k (global indices)")
+
+
+def test_compact_strided_outputs_and_guard_bands():
+    """Outputs are views into a wider cache buffer; bytes outside the views must stay untouched."""
+    p = W.random_problem(seed=8, lens=[64], rows=[1], keeps=[20], num_q_heads=4, num_kv_heads=2, head_dim=64, hidden=128)
+    keep_idx = np.sort(np.random.default_rng(1).choice(64, 20, replace=False)).astype(np.int32)
+    cache = torch.full((20 + 2, 2 * 2 + 1, 64), 7.0, dtype=torch.bfloat16, device="cuda")   # [tokens+guard, k|v|pad heads, d]
+    k_out, v_out = cache[1:21, 0:2], cache[1:21, 2:4]
+    buf = parity.to_device(p, flags=0)
+    buf.k_out, buf.v_out = k_out, v_out
+    buf.params.ko_stride_tok, buf.params.ko_stride_head = k_out.stride(0), k_out.stride(1)
+    buf.params.vo_stride_tok, buf.params.vo_stride_head = v_out.stride(0), v_out.stride(1)
+    buf.keep_idx[:20].copy_(torch.as_tensor(keep_idx))
+    buf.cu_keep.copy_(torch.tensor([0, 20], dtype=torch.int32))
+    buf.compact()
+    assert _sync_status(buf) == 0
+    ref = oracle.compact(keep_idx, np.array([0, 20], dtype=np.int32), p.cu_seqlens.numpy(), None, None, bf16_bits(p.k), bf16_bits(p.v))
+    parity.assert_bits_equal(k_out.contiguous(), ref["k"], "k view")
+    parity.assert_bits_equal(v_out.contiguous(), ref["v"], "v view")
+    host = cache.cpu().float()
+    assert (host[0] == 7).all() and (host[21] == 7).all() and (host[:, 4] == 7).all()
+
+
+def test_compact_reports_out_of_range_indices():
+    p = W.random_problem(seed=9, lens=[16], rows=[1], keeps=[4], num_q_heads=2, num_kv_heads=1, head_dim=64, hidden=64)
+    buf = parity.to_device(p, flags=0)
+    buf.keep_idx[:4].copy_(torch.tensor([0, 5, 99, -2], dtype=torch.int32))
+    buf.cu_keep.copy_(torch.tensor([0, 4], dtype=torch.int32))
+    buf.hidden_out.zero_()
+    buf.compact()
+    assert _sync_status(buf) & fastav.FASTAV_DEV_BAD_INDEX
+    out = buf.hidden_out.cpu()
+    assert torch.equal(out[1].view(torch.int16), p.hidden[5].view(torch.int16)) and (out[2:] == 0).all()
+
+
+# ---- fused prune ------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("lens,rows,keeps,hq,hkv,d,hid", [
+    ([9], [1], [4], 4, 2, 64, 64),
+    ([129, 0, 64], [4, 0, 1], [64, 0, 64], 8, 2, 64, 128),
+    ([1000, 7], [3, 2], [999, 1], 28, 4, 128, 256),
+    ([300], [64], [150], 8, 2, 128, 512),
+])
+@pytest.mark.parametrize("protect_rows", [True, False])
+def test_prune_small_problems(lens, rows, keeps, hq, hkv, d, hid, protect_rows):
+    p = W.random_problem(seed=len(lens) * 31 + hq, lens=lens, rows=rows, keeps=keeps, num_q_heads=hq, num_kv_heads=hkv,
+                         head_dim=d, hidden=hid, duplicate_keys=4)
+    p.protect_rows = protect_rows
+    buf = parity.to_device(p)
+    buf.prune()
+    torch.cuda.synchronize()
+    ref = parity.oracle_prune(p)
+    stats = parity.check_fused_against_oracle(p, buf, ref, what=f"lens={lens}")
+    assert stats["device_status"] == 0
+    # twice in a row: bit-identical everything
+    first = {k: getattr(buf, k).clone() for k in ("scores", "keep_idx", "hidden_out", "k_out", "v_out", "pos_out")}
+    buf.prune()
+    torch.cuda.synchronize()
+    for k, t in first.items():
+        assert torch.equal(t.view(torch.int32) if t.dtype == torch.float32 else t.view(torch.int16) if t.dtype == torch.bfloat16 else t,
+                           getattr(buf, k).view(torch.int32) if t.dtype == torch.float32 else getattr(buf, k).view(torch.int16) if t.dtype == torch.bfloat16 else getattr(buf, k)), k
+
+
+def test_prune_with_protect_mask_keeps_all_text_tokens():
+    w = W.WORKLOADS["c1_tiny"]
+    p = W.make_stage(w, 0)
+    protect = (p.modality == W.MOD_TEXT).to(torch.uint8)
+    buf = parity.to_device(p, protect=protect)
+    buf.prune()
+    torch.cuda.synchronize()
+    ref = parity.oracle_prune(p, protect=protect)
+    parity.check_fused_against_oracle(p, buf, ref, protect=protect, what="protect mask")
+    kept = set(buf.keep_idx.cpu().tolist())
+    assert set(torch.nonzero(protect).flatten().tolist()) <= kept
+
+
+def _run_workload_chain(name, stats_out=None):
+    """All stages of a workload; stage s+1 starts from the ORACLE's survivors of stage s."""
+    w = W.WORKLOADS[name]
+    hidden = pos = None
+    for si in range(len(w.stages)):
+        p = W.make_stage(w, si)
+        if si == 0:
+            hidden, pos = p.hidden, p.pos
+        buf = parity.to_device(p, hidden=hidden, pos=pos)
+        buf.prune()
+        torch.cuda.synchronize()
+        ref = parity.oracle_prune(p, hidden=hidden, pos=pos)
+        stats = parity.check_fused_against_oracle(p, buf, ref, hidden=hidden, pos=pos, what=f"{name} stage {si}")
+        assert stats["device_status"] == 0
+        got = buf.scores.cpu().numpy()
+        cu = p.cu_seqlens.numpy()
+        sums = np.add.reduceat(got, cu[:-1])
+        assert np.abs(sums - 1.0).max() < 1e-4
+        assert int(buf.cu_keep[-1]) == p.total_keep
+        if stats_out is not None:
+            stats_out.append(stats)
+        hidden = torch.as_tensor(ref["hidden"].view(np.int16)).view(torch.bfloat16)
+        pos = torch.as_tensor(ref["pos"])
+        del buf
+        torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("name", ["c1_tiny", "c2_global_2k", "c3_fine_chain"])
+def test_prune_workloads_small(name):
+    _run_workload_chain(name)
+
+
+@pytest.mark.parametrize("name", ["c4_long_av", "c5_ragged"])
+def test_prune_workloads_full_size(name):
+    stats = []
+    _run_workload_chain(name, stats)
+    print(name, stats)
