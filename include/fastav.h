@@ -163,6 +163,30 @@ int32_t fastav_prune(const fastav_params* params, const void* q, const int32_t* 
                      int32_t* keep_idx_out, int32_t* cu_keep_out, void* hidden_out, int32_t* pos_out, void* k_out,
                      void* v_out, void* workspace, size_t workspace_bytes, int32_t* device_status, void* stream);
 
+/*
+ * The same prune step for tensors that live in HOST memory (offloaded activations or KV cache):
+ * every data pointer of this call is a host pointer (pinned memory makes the copies asynchronous).
+ * The call enqueues host-to-device copies of the inputs, fastav_prune, and device-to-host copies
+ * of scores, keep_idx, cu_keep, the compacted tensors and the device status word (status_out,
+ * optional) on `stream`, staged through `device_arena`, a DEVICE buffer of at least
+ * fastav_host_arena_bytes() bytes, 256-byte aligned, owned by the caller.  Host outputs are valid
+ * once the stream has been synchronised.  Only packed layouts are accepted (token stride =
+ * heads * head_dim, head stride = head_dim; otherwise FASTAV_ERR_UNSUPPORTED).  The paper has no
+ * counterpart for this entry point; it computes exactly what fastav_prune computes.
+ */
+int32_t fastav_host_arena_bytes(const fastav_params* params, size_t* out_bytes);
+int32_t fastav_prune_host(const fastav_params* params, const void* q, const int32_t* q_idx, const int32_t* cu_qlens,
+                          const void* k, const void* v, const int32_t* cu_seqlens, const int32_t* keep_counts,
+                          const uint8_t* protect_opt, const void* hidden_in, const int32_t* pos_in, float* scores_out,
+                          int32_t* keep_idx_out, int32_t* cu_keep_out, void* hidden_out, int32_t* pos_out, void* k_out,
+                          void* v_out, int32_t* status_out, void* device_arena, size_t arena_bytes, void* stream);
+
+/*
+ * Number of kernels this library has launched in this process so far (a diagnostic counter; the
+ * only process-wide state the library has).  Benchmarks read it before and after a timed region.
+ */
+int64_t fastav_kernel_launches(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -57,6 +57,8 @@ def _u16_strided(a, name):
     a = np.asarray(a)
     if a.dtype != np.uint16 or a.ndim != 3:
         raise TypeError(f"{name}: expected a 3-d uint16 (bf16 bits) array")
+    if a.size == 0:  # numpy reports arbitrary strides for empty arrays
+        return a, a.shape[1] * a.shape[2], a.shape[2]
     if a.strides[2] != 2 or a.strides[0] % 2 or a.strides[1] % 2:
         raise ValueError(f"{name}: last axis must be contiguous")
     return a, a.strides[0] // 2, a.strides[1] // 2

@@ -1,5 +1,6 @@
 // C-ABI layer: argument validation, workspace carving and kernel dispatch.  See fastav.h for the
 // contract of every entry point; nothing here computes anything.
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -10,6 +11,7 @@ namespace fastav {
 namespace {
 
 thread_local char g_cuda_error[256] = "";
+std::atomic<long long> g_launches{0};
 
 int32_t cuda_failed(cudaError_t e) {
   std::snprintf(g_cuda_error, sizeof g_cuda_error, "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
@@ -127,6 +129,8 @@ int32_t check_compact_args(const fastav_params* p, const int32_t* keep_idx, cons
 
 }  // namespace
 
+void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
 Workspace plan_workspace(const fastav_params& p) {
   Workspace w;
   size_t off = 0;
@@ -169,6 +173,8 @@ const char* fastav_status_string(int32_t status) {
 }
 
 const char* fastav_last_cuda_error(void) { return g_cuda_error; }
+
+int64_t fastav_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
 
 int32_t fastav_workspace_bytes(const fastav_params* params, size_t* out_bytes) {
   int32_t rc = check_params(params);

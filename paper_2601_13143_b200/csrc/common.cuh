@@ -55,6 +55,9 @@ cudaError_t launch_compact(const Shapes& s, const int32_t* keep_idx, const int32
                            int32_t* pos_out, const void* k_in, void* k_out, const void* v_in, void* v_out,
                            int32_t* device_status, cudaStream_t stream);
 
+// Diagnostic launch counter (fastav_kernel_launches).
+void count_launches(int n);
+
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 }  // namespace fastav

@@ -112,6 +112,7 @@ cudaError_t launch_compact(const Shapes& s, const int32_t* keep_idx, const int32
   int blocks = kNumSMs * 8;
   if (blocks > s.total_keep) blocks = s.total_keep;
   compact_rows_kernel<<<blocks, kThreads, 0, stream>>>(s, t, keep_idx, cu_keep, cu_seqlens, device_status);
+  count_launches(1);
   return cudaGetLastError();
 }
 

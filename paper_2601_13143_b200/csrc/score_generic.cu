@@ -253,10 +253,12 @@ cudaError_t run(const Shapes& s, const Workspace& w, const uint16_t* q, const in
     const int warps = s.total_q * s.hq;
     score_merge_stats_kernel<<<(warps + 7) / 8, 256, 0, stream>>>(s, cu_qlens, cu_seqlens, stats, w.stat_tiles, lse);
     score_tile_accumulate_kernel<DIM><<<grid, kThreads, smem, stream>>>(s, q, q_idx, cu_qlens, k, cu_seqlens, lse, partial);
+    count_launches(3);
   }
   if (s.max_seqlen > 0) {
     const dim3 grid((s.max_seqlen + 255) / 256, s.batch);
     score_finalize_kernel<<<grid, 256, 0, stream>>>(s, cu_seqlens, cu_qlens, partial, scores_out);
+    count_launches(1);
   }
   return cudaGetLastError();
 }

@@ -191,6 +191,7 @@ cudaError_t launch_select(const Shapes& s, const Workspace& w, const float* scor
                                                                     cu_qlens, keep_idx, cu_keep,
                                                                     reinterpret_cast<unsigned*>(ws + w.keys_off), device_status);
   }
+  count_launches(1);
   return cudaGetLastError();
 }
 

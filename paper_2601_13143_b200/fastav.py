@@ -30,7 +30,8 @@ FASTAV_ERR_CUDA = -4
 FASTAV_ERR_TIMEOUT = -5
 
 EXPORTS = ("fastav_version", "fastav_status_string", "fastav_last_cuda_error", "fastav_workspace_bytes",
-           "fastav_score", "fastav_select", "fastav_compact", "fastav_prune")
+           "fastav_score", "fastav_select", "fastav_compact", "fastav_prune", "fastav_host_arena_bytes",
+           "fastav_prune_host", "fastav_kernel_launches")
 
 
 class fastav_params(ctypes.Structure):
@@ -94,6 +95,12 @@ def library() -> ctypes.CDLL:
         lib.fastav_prune.restype = ctypes.c_int32
         lib.fastav_prune.argtypes = [pp, vp, i32p, i32p, vp, vp, i32p, i32p, vp, vp, i32p, vp, i32p, i32p, vp, i32p,
                                      vp, vp, vp, ctypes.c_size_t, i32p, vp]
+        lib.fastav_host_arena_bytes.restype = ctypes.c_int32
+        lib.fastav_host_arena_bytes.argtypes = [pp, ctypes.POINTER(ctypes.c_size_t)]
+        lib.fastav_prune_host.restype = ctypes.c_int32
+        lib.fastav_prune_host.argtypes = [pp, vp, i32p, i32p, vp, vp, i32p, i32p, vp, vp, i32p, vp, i32p, i32p, vp, i32p,
+                                          vp, vp, i32p, vp, ctypes.c_size_t, vp]
+        lib.fastav_kernel_launches.restype = ctypes.c_int64
         _lib = lib
     return _lib
 
@@ -188,6 +195,32 @@ def fastav_prune(params, q, q_idx, cu_qlens, k, v, cu_seqlens, keep_counts, prot
                                   _p(keep_counts), _p(protect_opt), _p(hidden_in), _p(pos_in), _p(scores_out),
                                   _p(keep_idx_out), _p(cu_keep_out), _p(hidden_out), _p(pos_out), _p(k_out), _p(v_out),
                                   ws, ws_bytes, _p(device_status), _stream(stream)), "fastav_prune")
+
+
+def fastav_kernel_launches() -> int:
+    return int(library().fastav_kernel_launches())
+
+
+def fastav_host_arena_bytes(params: fastav_params) -> int:
+    out = ctypes.c_size_t(0)
+    _check(library().fastav_host_arena_bytes(ctypes.byref(params), ctypes.byref(out)), "fastav_host_arena_bytes")
+    return int(out.value)
+
+
+def fastav_prune_host(params, q, q_idx, cu_qlens, k, v, cu_seqlens, keep_counts, protect_opt, hidden_in, pos_in, scores_out,
+                      keep_idx_out, cu_keep_out, hidden_out, pos_out, k_out, v_out, status_out, device_arena,
+                      stream=None) -> None:
+    """All tensors are HOST tensors (pinned for asynchronous copies) except ``device_arena``."""
+    for t in (q, q_idx, cu_qlens, k, v, cu_seqlens, keep_counts, protect_opt, hidden_in, pos_in, scores_out, keep_idx_out,
+              cu_keep_out, hidden_out, pos_out, k_out, v_out, status_out):
+        if t is not None and (t.is_cuda or not t.is_contiguous()):
+            raise ValueError("fastav_prune_host takes contiguous host tensors")
+    _check(library().fastav_prune_host(ctypes.byref(params), _p(q), _p(q_idx), _p(cu_qlens), _p(k), _p(v), _p(cu_seqlens),
+                                       _p(keep_counts), _p(protect_opt), _p(hidden_in), _p(pos_in), _p(scores_out),
+                                       _p(keep_idx_out), _p(cu_keep_out), _p(hidden_out), _p(pos_out), _p(k_out), _p(v_out),
+                                       _p(status_out), _p(device_arena),
+                                       ctypes.c_size_t(device_arena.numel() * device_arena.element_size()),
+                                       _stream(stream)), "fastav_prune_host")
 
 
 # ---- convenience: buffers for one prune call --------------------------------------------------
