@@ -1,0 +1,409 @@
+#!/usr/bin/env python
+"""Benchmark of the FastAV prune step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+A "step" is one pass of the whole hot path over one batch of synthetic input: every pruning stage
+of the workload (score -> select -> compact, fused in ``fastav_prune``), stage s+1 running on the
+survivors of stage s.  The default workload is the long audio-video clip (4 x 16384 tokens,
+Mistral-7B shapes, global keep 40 % then fine keep 70 %), the configuration whose inputs exceed L2
+and on which the HBM-roofline target is quoted.  Prints ONE JSON line (rank 0).
+
+Multi-GPU: the path does not shard (per-sequence softmax, top-k and gather; no exchange step), so
+``--gpus N`` under torchrun runs N independent replicas, one per GPU, and reports the aggregate.
+
+``--impl reference`` times the CPU oracle (the plain definition the kernels are checked against) on
+the host cores, on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2601_13143_b200 import workloads as W  # noqa: E402
+from paper_2601_13143_b200 import flops as F  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_HBM_GBS = 6650.0
+METRIC = "prune-step tokens/s"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (None until a capture of that kernel exists).
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "sm_max_mhz": float(d.get("sm_max_mhz", 1965.0)), "source": "measured"}
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "sm_max_mhz": 1965.0, "source": "fallback"}
+
+
+# ---- algorithmic bytes (what the method itself must move) ---------------------------------------
+
+def stage_bytes(m: W.ModelShape, n_tokens: int, n_rows: int, n_keep: int) -> dict:
+    kv_row = m.num_kv_heads * m.head_dim * 2
+    score = n_tokens * kv_row + n_rows * m.num_q_heads * m.head_dim * 2 + 4 * n_tokens
+    select = 4 * n_tokens + 4 * n_keep
+    compact = n_keep * (4 + 2 * (m.hidden * 2 + 2 * kv_row + 4))
+    return {"score": score, "select": select, "compact": compact, "total": score + select + compact}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=lambda: self.lines.extend(self.proc.stdout), daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+            self.thread.join(timeout=5)
+
+    def summary(self) -> dict:
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def build_chain(w: W.Workload, device):
+    """Device buffers for every stage; stage s+1 reads the compacted hidden states / positions of stage s."""
+    from paper_2601_13143_b200 import fastav
+    stages, prev = [], None
+    for si in range(len(w.stages)):
+        p = W.make_stage(w, si)
+        hidden = p.hidden.to(device) if si == 0 else prev.hidden_out
+        pos = p.pos.to(device) if si == 0 else prev.pos_out
+        lens = (p.cu_seqlens[1:] - p.cu_seqlens[:-1]).tolist()
+        rows = (p.cu_qlens[1:] - p.cu_qlens[:-1]).tolist()
+        flags = fastav.FASTAV_CAUSAL | fastav.FASTAV_PROTECT_QUERY_ROWS
+        buf = fastav.make_buffers(q=p.q.to(device), q_idx=p.q_idx.to(device), cu_qlens=p.cu_qlens.to(device), k=p.k.to(device),
+                                  v=p.v.to(device), cu_seqlens=p.cu_seqlens.to(device), keep_counts=p.keep_counts.to(device),
+                                  hidden=hidden, pos=pos, softmax_scale=p.softmax_scale, flags=flags, lens=lens, rows=rows,
+                                  keeps=p.keep_counts.tolist())
+        stages.append((p, buf))
+        prev = buf
+    return stages
+
+
+def host_chain(w: W.Workload, device):
+    """Pinned host tensors + device arena per stage for the end-to-end (host-buffer) measurement."""
+    from paper_2601_13143_b200 import fastav
+    pin = lambda t: t.contiguous().pin_memory()
+    out, prev = [], None
+    for si in range(len(w.stages)):
+        p = W.make_stage(w, si)
+        m = p.model
+        lens = (p.cu_seqlens[1:] - p.cu_seqlens[:-1]).tolist()
+        rows = (p.cu_qlens[1:] - p.cu_qlens[:-1]).tolist()
+        keeps = p.keep_counts.tolist()
+        n, kk = sum(lens), sum(keeps)
+        params = fastav.make_params(batch=len(lens), total_tokens=n, max_seqlen=max(lens), total_q=sum(rows), max_qlen=max(rows),
+                                    total_keep=kk, max_keep=max(keeps), num_q_heads=m.num_q_heads, num_kv_heads=m.num_kv_heads,
+                                    head_dim=m.head_dim, hidden=m.hidden, softmax_scale=p.softmax_scale,
+                                    flags=fastav.FASTAV_CAUSAL | fastav.FASTAV_PROTECT_QUERY_ROWS)
+        h = {"params": params, "q": pin(p.q), "q_idx": pin(p.q_idx), "cu_qlens": pin(p.cu_qlens), "k": pin(p.k), "v": pin(p.v),
+             "cu_seqlens": pin(p.cu_seqlens), "keep_counts": pin(p.keep_counts),
+             "hidden": pin(p.hidden) if si == 0 else prev["hidden_out"], "pos": pin(p.pos) if si == 0 else prev["pos_out"],
+             "scores": pin(torch.empty(n, dtype=torch.float32)), "keep_idx": pin(torch.empty(max(kk, 1), dtype=torch.int32)),
+             "cu_keep": pin(torch.empty(len(lens) + 1, dtype=torch.int32)),
+             "hidden_out": pin(torch.empty(kk, m.hidden, dtype=torch.bfloat16)), "pos_out": pin(torch.empty(kk, dtype=torch.int32)),
+             "k_out": pin(torch.empty(kk, m.num_kv_heads, m.head_dim, dtype=torch.bfloat16)),
+             "v_out": pin(torch.empty(kk, m.num_kv_heads, m.head_dim, dtype=torch.bfloat16)),
+             "status": pin(torch.zeros(1, dtype=torch.int32)),
+             "arena": torch.empty(fastav.fastav_host_arena_bytes(params), dtype=torch.uint8, device=device)}
+        ins = ("q", "q_idx", "cu_qlens", "k", "v", "cu_seqlens", "keep_counts", "hidden", "pos")
+        outs = ("scores", "keep_idx", "cu_keep", "hidden_out", "pos_out", "k_out", "v_out", "status")
+        h["h2d"] = sum(h[x].numel() * h[x].element_size() for x in ins)
+        h["d2h"] = sum(h[x].numel() * h[x].element_size() for x in outs)
+        out.append(h)
+        prev = h
+    return out
+
+
+def run_host_step(chain):
+    from paper_2601_13143_b200 import fastav
+    for h in chain:
+        fastav.fastav_prune_host(h["params"], h["q"], h["q_idx"], h["cu_qlens"], h["k"], h["v"], h["cu_seqlens"], h["keep_counts"],
+                                 None, h["hidden"], h["pos"], h["scores"], h["keep_idx"], h["cu_keep"], h["hidden_out"],
+                                 h["pos_out"], h["k_out"], h["v_out"], h["status"], h["arena"])
+
+
+def oracle_sample(w: W.Workload):
+    """Bounded sample for the CPU legs: the first sequence of every stage."""
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from conftest import bf16_bits
+    sample = []
+    for si in range(len(w.stages)):
+        p = W.make_stage(w, si)
+        n, r = int(p.cu_seqlens[1]), int(p.cu_qlens[1])
+        hidden = p.hidden[:n] if p.hidden is not None else torch.zeros(n, p.model.hidden, dtype=torch.bfloat16)
+        pos = p.pos[:n] if p.pos is not None else torch.arange(n, dtype=torch.int32)
+        sample.append(dict(q=bf16_bits(p.q[:r]), k=bf16_bits(p.k[:n]), v=bf16_bits(p.v[:n]), hidden=bf16_bits(hidden), pos=pos.numpy(),
+                           cu_seqlens=[0, n], cu_qlens=[0, r], q_idx=p.q_idx[:r].numpy(), keep_counts=[int(p.keep_counts[0])],
+                           scale=p.softmax_scale, causal=p.causal, tokens=n))
+    return sample
+
+
+def run_oracle_sample(sample) -> None:
+    import oracle
+    for s in sample:
+        oracle.prune(s["q"], s["k"], s["v"], s["hidden"], s["pos"], s["cu_seqlens"], s["cu_qlens"], s["q_idx"], s["keep_counts"],
+                     s["scale"], s["causal"], protect_rows=True)
+
+
+def workload_config(w: W.Workload, lens) -> dict:
+    m = w.model
+    return {"workload": w.name, "description": w.description, "batch": w.batch, "tokens_per_stage": [sum(x) for x in lens],
+            "stages": [{"layer": s.layer, "scored_rows": s.rows, "keep": s.keep if s.keep is not None else list(w.keep_range)}
+                       for s in w.stages],
+            "shapes": {"name": m.name, "q_heads": m.num_q_heads, "kv_heads": m.num_kv_heads, "head_dim": m.head_dim,
+                       "hidden": m.hidden}}
+
+
+def flops_removed(w: W.Workload, lens) -> dict:
+    """Prefill FLOPs the workload's schedule removes, summed over the batch."""
+    m = w.model
+    full = pruned = 0
+    for b in range(w.batch):
+        sched = {st.layer: lens[si + 1][b] for si, st in enumerate(w.stages)}
+        r = F.schedule_flops(lens[0][b], sched, m.num_layers, m.hidden, m.ffn)
+        full += r["full"]
+        pruned += r["pruned"]
+    return {"removed_tflop": (full - pruned) / 1e12, "relative_to_100": 100.0 * pruned / full}
+
+
+def main_reference(args, w, lens):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    sample = oracle_sample(w)
+    tokens = sum(s["tokens"] for s in sample)
+    for _ in range(args.warmup):
+        run_oracle_sample(sample)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        run_oracle_sample(sample)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = tokens / dt
+    desc = f"first sequence of each stage ({tokens} tokens per step) of {w.name}"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic", "config": workload_config(w, lens),
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": oracle.max_threads(), "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="c4_long_av", choices=list(W.WORKLOAD_ORDER))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    w = W.WORKLOADS[args.workload]
+    lens = W.stage_lengths(w)
+    if args.impl == "reference":
+        return main_reference(args, w, lens)
+
+    from paper_2601_13143_b200 import fastav
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the prune path has no CPU fallback")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    fastav.library()
+    stages = build_chain(w, device)
+    stream = torch.cuda.current_stream()
+    tokens_per_step = sum(sum(x) for x in lens[:-1])
+    bytes_per_stage = [stage_bytes(p.model, p.total_tokens, int(p.cu_qlens[-1]), p.total_keep) for p, _ in stages]
+    bytes_per_step = sum(b["total"] for b in bytes_per_stage)
+    needs_flush = bytes_per_stage[0]["total"] < 2 * L2_BYTES
+    flush_buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=device) if needs_flush else None
+
+    def step():
+        for _, buf in stages:
+            buf.prune(stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    status = sum(int(buf.device_status.cpu()) for _, buf in stages)
+
+    # ---- the timed region: exactly K steps, device time, max over ranks ----
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    stops = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    launches0 = fastav.fastav_kernel_launches()
+    barrier()
+    with ClockSampler(local) as clocks:
+        for i in range(args.steps):
+            if flush_buf is not None:
+                flush_buf.fill_(i & 0xFF)       # evict the inputs from L2 (outside the per-step events)
+            starts[i].record(stream)
+            step()
+            stops[i].record(stream)
+        torch.cuda.synchronize()
+    barrier()
+    launches = fastav.fastav_kernel_launches() - launches0
+    step_ms = [a.elapsed_time(b) for a, b in zip(starts, stops)]
+    total_ms = sum(step_ms)
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * tokens_per_step / (ms_per_step * 1e-3)
+
+    # ---- per-kernel times of the same steps (separate entry points, events in between) ----
+    phase_ms = [{"score": 0.0, "select": 0.0, "compact": 0.0} for _ in stages]
+    reps = min(args.steps, 10)
+    for i in range(reps):
+        for si, (_, buf) in enumerate(stages):
+            if flush_buf is not None:
+                flush_buf.fill_(i & 0xFF)
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            ev[0].record(stream); buf.score(stream)
+            ev[1].record(stream); buf.select(stream)
+            ev[2].record(stream); buf.compact(stream)
+            ev[3].record(stream)
+            torch.cuda.synchronize()
+            for j, name in enumerate(("score", "select", "compact")):
+                phase_ms[si][name] += ev[j].elapsed_time(ev[j + 1]) / reps
+
+    peaks = measured_peaks()
+    phases = []
+    for si, ((p, _), b, t) in enumerate(zip(stages, bytes_per_stage, phase_ms)):
+        rows_heads_tokens = sum(int(p.cu_qlens[i + 1] - p.cu_qlens[i]) * int(p.cu_seqlens[i + 1] - p.cu_seqlens[i])
+                                for i in range(p.batch)) * p.model.num_q_heads
+        phases.append({"stage": si, "tokens": p.total_tokens, "ms": {k: round(v, 5) for k, v in t.items()},
+                       "gbs": {k: round(b[k] / (t[k] * 1e-3) / 1e9, 1) if t[k] > 0 else None for k in t},
+                       "bytes": b, "score_exp2_per_sweep": rows_heads_tokens})
+    # dominant kernel of the step
+    dom_stage, dom_name = max(((si, name) for si in range(len(stages)) for name in ("score", "select", "compact")),
+                              key=lambda x: phase_ms[x[0]][x[1]])
+    dom_ms = phase_ms[dom_stage][dom_name]
+    dom_bytes = bytes_per_stage[dom_stage][dom_name]
+    achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
+    roofline = {"kernel": f"{dom_name} (stage {dom_stage})", "bound": "hbm", "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"],
+                "unit": "GB/s", "frac": round(achieved / peaks["hbm_gbs"], 4), "of": peaks["source"],
+                "traffic": NCU_TRAFFIC_BYTES.get(f"{w.name}:{dom_stage}:{dom_name}"), "algorithmic_bytes": dom_bytes,
+                "ms": round(dom_ms, 5)}
+    step_gbs = bytes_per_step / (ms_per_step * 1e-3) / 1e9
+    compact_rooflines = [{"stage": si, "achieved": ph["gbs"]["compact"], "frac": round(ph["gbs"]["compact"] / peaks["hbm_gbs"], 4)}
+                         for si, ph in enumerate(phases) if ph["gbs"]["compact"]]
+
+    # ---- end to end: host buffers through fastav_prune_host, copies inside the timed region ----
+    e2e = None
+    if not args.no_e2e:
+        chain = host_chain(w, device)
+        e2e_steps = min(args.steps, 5)
+        run_host_step(chain)
+        torch.cuda.synchronize()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(e2e_steps):
+            run_host_step(chain)
+        b.record(stream)
+        torch.cuda.synchronize()
+        barrier()
+        e2e_ms = a.elapsed_time(b) / e2e_steps
+        if dist is not None:
+            t = torch.tensor([e2e_ms], dtype=torch.float64, device=device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        e2e = {"value": world * tokens_per_step / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms, "steps": e2e_steps,
+               "h2d_bytes_per_step": sum(h["h2d"] for h in chain), "d2h_bytes_per_step": sum(h["d2h"] for h in chain),
+               "api": "fastav_prune_host (pinned host buffers)"}
+        del chain
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        sample = oracle_sample(w)
+        t0 = time.perf_counter()
+        run_oracle_sample(sample)
+        dt = time.perf_counter() - t0
+        stoks = sum(s["tokens"] for s in sample)
+        cpu = {"value": stoks / dt, "unit": "tokens/s", "cores": oracle.max_threads(), "kind": "oracle", "seconds": round(dt, 3),
+               "sample": f"first sequence of each stage ({stoks} tokens) of {w.name}, one pass"}
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic", "config": {**workload_config(w, lens), "parallelism": "replicas" if world > 1 else "single",
+                                            "l2": "L2 flushed between steps" if needs_flush else "inputs larger than L2"},
+            "step_hbm": {"algorithmic_bytes": bytes_per_step, "gbs": round(step_gbs, 1), "frac_of_peak": round(step_gbs / peaks["hbm_gbs"], 4),
+                         "frac_of_nominal_8tbs": round(step_gbs / 8000.0, 4), "of": peaks["source"]},
+            "roofline": roofline, "compact_roofline": compact_rooflines, "phases": phases,
+            "prefill_flops": flops_removed(w, lens), "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": launches,
+            "device_status": status, "clocks": clocks.summary()}))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -312,3 +312,29 @@ def test_prune_workloads_full_size(name):
     stats = []
     _run_workload_chain(name, stats)
     print(name, stats)
+
+
+def test_prune_host_buffers_match_oracle():
+    """The host-buffer entry point computes the same step (copies in, fused prune, copies out)."""
+    p = W.make_stage(W.WORKLOADS["c1_tiny"], 0)
+    m = p.model
+    n, kk = p.total_tokens, p.total_keep
+    params = fastav.make_params(batch=1, total_tokens=n, max_seqlen=n, total_q=4, max_qlen=4, total_keep=kk, max_keep=kk,
+                                num_q_heads=m.num_q_heads, num_kv_heads=m.num_kv_heads, head_dim=m.head_dim, hidden=m.hidden,
+                                softmax_scale=p.softmax_scale, flags=parity.flags_of(p))
+    pin = lambda t: t.contiguous().pin_memory()
+    out = dict(scores=pin(torch.empty(n)), keep_idx=pin(torch.empty(kk, dtype=torch.int32)), cu_keep=pin(torch.empty(2, dtype=torch.int32)),
+               hidden=pin(torch.empty(kk, m.hidden, dtype=torch.bfloat16)), pos=pin(torch.empty(kk, dtype=torch.int32)),
+               k=pin(torch.empty(kk, m.num_kv_heads, m.head_dim, dtype=torch.bfloat16)),
+               v=pin(torch.empty(kk, m.num_kv_heads, m.head_dim, dtype=torch.bfloat16)), status=pin(torch.full((1,), -1, dtype=torch.int32)))
+    arena = torch.empty(fastav.fastav_host_arena_bytes(params), dtype=torch.uint8, device="cuda")
+    fastav.fastav_prune_host(params, pin(p.q), pin(p.q_idx), pin(p.cu_qlens), pin(p.k), pin(p.v), pin(p.cu_seqlens),
+                             pin(p.keep_counts), None, pin(p.hidden), pin(p.pos), out["scores"], out["keep_idx"], out["cu_keep"],
+                             out["hidden"], out["pos"], out["k"], out["v"], out["status"], arena)
+    torch.cuda.synchronize()
+    ref = parity.oracle_prune(p)
+    parity.assert_scores_close(out["scores"], ref["scores"], "host")
+    assert int(out["status"]) == 0 and out["cu_keep"].tolist() == [0, kk]
+    assert out["keep_idx"].tolist() == ref["keep_idx"].tolist()
+    for name in ("hidden", "pos", "k", "v"):
+        parity.assert_bits_equal(out[name], ref[name], "host " + name)
