@@ -182,6 +182,37 @@ int32_t fastav_prune_host(const fastav_params* params, const void* q, const int3
                           void* v_out, int32_t* status_out, void* device_arena, size_t arena_bytes, void* stream);
 
 /*
+ * fastav_select without any caller-provided scratch.  The paper has no counterpart for this
+ * entry point: it exists for callers that cannot allocate device memory at the point where they
+ * prune -- a plug-in running inside a host application that hands it input and output tensors
+ * only, a real-time loop in which cudaMalloc's implicit synchronisation is not acceptable, a
+ * process whose memory pool is fixed and fully assigned at start-up.  fastav_select needs a
+ * workspace (one 32-bit key per token) whenever a sequence is too long for shared memory; here
+ * the keys always go to an array built into the library, so the call takes no workspace and
+ * never calls cudaMalloc, cudaFree or any routine that allocates.
+ *
+ * Limits and rules
+ *   - total_tokens <= FASTAV_NOALLOC_MAX_TOKENS, else FASTAV_ERR_UNSUPPORTED (nothing enqueued).
+ *     The array costs 4 * FASTAV_NOALLOC_MAX_TOKENS bytes (4 MiB) of device memory on every GPU
+ *     on which the library is loaded, until the process exits.
+ *   - The first call on each device looks up the array's device address (a runtime query, made
+ *     with that device current, cached afterwards).  Make that first call during set-up, before
+ *     any stream capture.
+ *   - All calls on a device share the one array.  Two calls whose kernels can overlap on the GPU
+ *     (different streams, no dependency between them) race on it and both results are undefined;
+ *     calls on one stream, or otherwise ordered, are fine.  Nothing has to be cleared between
+ *     calls: each call overwrites every key before reading it.
+ *   - Of params only batch, total_tokens, max_seqlen, total_q, total_keep and flags are read.
+ * Arguments, outputs, tie rule and device status bits are exactly those of fastav_select, and
+ * the two produce identical keep_idx_out / cu_keep_out.
+ */
+#define FASTAV_NOALLOC_MAX_TOKENS (1 << 20)
+int32_t fastav_select_noalloc(const fastav_params* params, const float* scores, const int32_t* cu_seqlens,
+                              const int32_t* keep_counts, const uint8_t* protect_opt, const int32_t* q_idx,
+                              const int32_t* cu_qlens, int32_t* keep_idx_out, int32_t* cu_keep_out,
+                              int32_t* device_status, void* stream);
+
+/*
  * Number of kernels this library has launched in this process so far (a diagnostic counter; the
  * only process-wide state the library has).  Benchmarks read it before and after a timed region.
  */

@@ -7,6 +7,8 @@
 // (k - #above) keys equal to T: ties go to the lower index and survivors come out ascending, which
 // is exactly the order the gather that follows needs.  Integer work throughout: the result is a
 // unique function of the fp32 score bits.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace fastav {
@@ -195,4 +197,65 @@ cudaError_t launch_select(const Shapes& s, const Workspace& w, const float* scor
   return cudaGetLastError();
 }
 
+// ---- fastav_select_noalloc: the same selection with its scratch inside the library ----------
+//
+// The radix select keeps one 32-bit key per token.  fastav_select puts them in shared memory or in
+// the caller's workspace; this variant always puts them in the array below, so a caller that owns
+// no device scratch (and may not obtain any) can still run the step.  The array lives in every
+// CUDA context that loads the library, from load to exit.
+namespace {
+
+static __device__ __align__(256) unsigned g_noalloc_keys[FASTAV_NOALLOC_MAX_TOKENS];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+unsigned* g_noalloc_ptr[kMaxDevices] = {};  // device address of g_noalloc_keys, per device ordinal
+
+// Device address of the scratch array on the current device.  In host code `g_noalloc_keys` is only
+// a handle for the symbol, not an address a kernel may use: the runtime translates it, once per
+// device, with that device current.
+cudaError_t noalloc_scratch(unsigned** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (!g_noalloc_ptr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_noalloc_keys);
+    if (e != cudaSuccess) return e;
+    g_noalloc_ptr[dev] = static_cast<unsigned*>(p);
+  }
+  *out = g_noalloc_ptr[dev];
+  return cudaSuccess;
+}
+
+}  // namespace
 }  // namespace fastav
+
+extern "C" int32_t fastav_select_noalloc(const fastav_params* p, const float* scores, const int32_t* cu_seqlens,
+                                         const int32_t* keep_counts, const uint8_t* protect_opt, const int32_t* q_idx,
+                                         const int32_t* cu_qlens, int32_t* keep_idx_out, int32_t* cu_keep_out,
+                                         int32_t* device_status, void* stream) {
+  using namespace fastav;
+  if (!p || p->batch < 1 || p->total_tokens < 0 || p->max_seqlen < 0 || p->max_seqlen > p->total_tokens ||
+      p->total_keep < 0 || p->total_keep > p->total_tokens || p->total_q < 0)
+    return FASTAV_ERR_INVALID_ARG;
+  if (p->total_tokens > FASTAV_NOALLOC_MAX_TOKENS) return FASTAV_ERR_UNSUPPORTED;  // beyond the built-in scratch
+  if (!cu_seqlens || !keep_counts || !cu_keep_out) return FASTAV_ERR_INVALID_ARG;
+  if (p->total_tokens > 0 && !scores) return FASTAV_ERR_INVALID_ARG;
+  if (p->total_keep > 0 && !keep_idx_out) return FASTAV_ERR_INVALID_ARG;
+  if ((p->flags & FASTAV_PROTECT_QUERY_ROWS) && (!cu_qlens || (p->total_q > 0 && !q_idx))) return FASTAV_ERR_INVALID_ARG;
+  unsigned* keys = nullptr;
+  if (noalloc_scratch(&keys) != cudaSuccess || !keys) return FASTAV_ERR_CUDA;
+  Shapes s{};
+  s.batch = p->batch; s.total_tokens = p->total_tokens; s.max_seqlen = p->max_seqlen;
+  s.total_q = p->total_q; s.max_qlen = p->max_qlen; s.total_keep = p->total_keep; s.max_keep = p->max_keep;
+  s.flags = p->flags;
+  // Every key a block reads was written by that block earlier in the same launch, so what an
+  // earlier call left in the array never matters and nothing has to be cleared.
+  select_topk_kernel<false><<<s.batch, kThreads, sizeof(SelectShared), static_cast<cudaStream_t>(stream)>>>(
+      s, scores, cu_seqlens, keep_counts, protect_opt, q_idx, cu_qlens, keep_idx_out, cu_keep_out, keys, device_status);
+  count_launches(1);
+  return cudaGetLastError() == cudaSuccess ? FASTAV_OK : FASTAV_ERR_CUDA;
+}

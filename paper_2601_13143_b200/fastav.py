@@ -31,7 +31,7 @@ FASTAV_ERR_TIMEOUT = -5
 
 EXPORTS = ("fastav_version", "fastav_status_string", "fastav_last_cuda_error", "fastav_workspace_bytes",
            "fastav_score", "fastav_select", "fastav_compact", "fastav_prune", "fastav_host_arena_bytes",
-           "fastav_prune_host", "fastav_kernel_launches")
+           "fastav_prune_host", "fastav_kernel_launches", "fastav_select_noalloc")
 
 
 class fastav_params(ctypes.Structure):
@@ -101,6 +101,8 @@ def library() -> ctypes.CDLL:
         lib.fastav_prune_host.argtypes = [pp, vp, i32p, i32p, vp, vp, i32p, i32p, vp, vp, i32p, vp, i32p, i32p, vp, i32p,
                                           vp, vp, i32p, vp, ctypes.c_size_t, vp]
         lib.fastav_kernel_launches.restype = ctypes.c_int64
+        lib.fastav_select_noalloc.restype = ctypes.c_int32
+        lib.fastav_select_noalloc.argtypes = [pp, vp, i32p, i32p, vp, i32p, i32p, i32p, i32p, i32p, vp]
         _lib = lib
     return _lib
 
@@ -178,6 +180,19 @@ def fastav_select(params, scores, cu_seqlens, keep_counts, protect_opt, q_idx, c
     _check(library().fastav_select(ctypes.byref(params), _p(scores), _p(cu_seqlens), _p(keep_counts), _p(protect_opt),
                                    _p(q_idx), _p(cu_qlens), _p(keep_idx_out), _p(cu_keep_out), ws, ws_bytes,
                                    _p(device_status), _stream(stream)), "fastav_select")
+
+
+NOALLOC_MAX_TOKENS = 1 << 20
+
+
+def fastav_select_noalloc(params, scores, cu_seqlens, keep_counts, protect_opt, q_idx, cu_qlens, keep_idx_out, cu_keep_out,
+                          device_status=None, stream=None) -> None:
+    """``fastav_select`` for callers that cannot allocate device memory: no workspace argument, the
+    keys live in an array inside the library (at most ``NOALLOC_MAX_TOKENS`` tokens per call; calls
+    that overlap on the GPU race on it)."""
+    _check(library().fastav_select_noalloc(ctypes.byref(params), _p(scores), _p(cu_seqlens), _p(keep_counts), _p(protect_opt),
+                                           _p(q_idx), _p(cu_qlens), _p(keep_idx_out), _p(cu_keep_out), _p(device_status),
+                                           _stream(stream)), "fastav_select_noalloc")
 
 
 def fastav_compact(params, keep_idx, cu_keep, cu_seqlens, hidden_in=None, hidden_out=None, pos_in=None, pos_out=None,
