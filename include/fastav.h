@@ -53,6 +53,13 @@ extern "C" {
 #define FASTAV_PROTECT_QUERY_ROWS 2u  /* the scored rows' tokens always survive (and count toward k_b) */
 #define FASTAV_KEEP_IDX_GLOBAL 4u     /* keep_idx holds indices into the packed batch, not sequence-local ones */
 
+/* Diagnostics: force one implementation of fastav_score instead of the shape-based choice.  A forced
+ * path that does not support the shapes makes the call fail with FASTAV_ERR_UNSUPPORTED. */
+#define FASTAV_SCORE_PATH_GENERIC 0x100u /* CUDA-core tiles, any shape */
+#define FASTAV_SCORE_PATH_NARROW 0x200u  /* matrix-vector path, max_qlen <= 4 */
+#define FASTAV_SCORE_PATH_WIDE 0x300u    /* tensor-core path */
+#define FASTAV_SCORE_PATH_MASK 0x300u
+
 /* bits OR-ed into *device_status */
 #define FASTAV_DEV_K_CLAMPED 1        /* some keep_counts[b] was outside [0, n_b] and was clamped */
 #define FASTAV_DEV_PROTECT_OVERFLOW 2 /* more protected tokens than k_b: the lowest-index ones were kept */

@@ -140,15 +140,29 @@ Workspace plan_workspace(const fastav_params& p) {
   w.stats_off = carve(rows_heads * (size_t)w.stat_tiles * sizeof(float2));
   w.lse_off = carve(rows_heads * sizeof(float));
   w.partial_off = carve((size_t)p.num_kv_heads * p.total_tokens * sizeof(float));
-  w.logits_off = carve(0);
+  const bool narrow = p.max_qlen >= 1 && p.max_qlen <= kNarrowMaxRows;
+  w.logits_off = carve(narrow ? (size_t)p.num_q_heads * p.max_qlen * p.total_tokens * sizeof(float) : 0);
   w.keys_off = carve((size_t)p.total_tokens * sizeof(uint32_t));
   w.total = off;
   return w;
 }
 
+// A forced score path (FASTAV_SCORE_PATH_*) must support the shapes; the shape-based choice always does.
+bool score_path_ok(const Shapes& s) {
+  const unsigned forced = s.flags & FASTAV_SCORE_PATH_MASK;
+  if (forced == FASTAV_SCORE_PATH_NARROW) return score_narrow_applies(s);
+  if (forced == FASTAV_SCORE_PATH_WIDE) return false;
+  return true;
+}
+
 cudaError_t launch_score(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
                          const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
                          unsigned char* ws, cudaStream_t stream) {
+  const unsigned forced = s.flags & FASTAV_SCORE_PATH_MASK;
+  if (forced == FASTAV_SCORE_PATH_GENERIC) return launch_score_generic(s, w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out, ws, stream);
+  if (score_narrow_applies(s) && (forced == 0 || forced == FASTAV_SCORE_PATH_NARROW))
+    return launch_score_narrow(s, w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out, ws, stream);
+  if (forced != 0) return cudaErrorNotSupported;
   return launch_score_generic(s, w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out, ws, stream);
 }
 
@@ -194,6 +208,7 @@ int32_t fastav_score(const fastav_params* params, const void* q, const int32_t* 
   if ((rc = check_score_args(params, q, q_idx, cu_qlens, k, cu_seqlens, scores_out)) != FASTAV_OK) return rc;
   const Workspace w = plan_workspace(*params);
   if ((rc = check_workspace(w, workspace, workspace_bytes)) != FASTAV_OK) return rc;
+  if (!score_path_ok(make_shapes(*params))) return FASTAV_ERR_UNSUPPORTED;
   if (params->total_tokens == 0) return FASTAV_OK;
   const cudaError_t e = launch_score(make_shapes(*params), w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out,
                                      static_cast<unsigned char*>(workspace), static_cast<cudaStream_t>(stream));
@@ -245,6 +260,7 @@ int32_t fastav_prune(const fastav_params* params, const void* q, const int32_t* 
   const Workspace w = plan_workspace(*params);
   if ((rc = check_workspace(w, workspace, workspace_bytes)) != FASTAV_OK) return rc;
   const Shapes s = make_shapes(*params);
+  if (!score_path_ok(s)) return FASTAV_ERR_UNSUPPORTED;
   unsigned char* ws = static_cast<unsigned char*>(workspace);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e = cudaSuccess;

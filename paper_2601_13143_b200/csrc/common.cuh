@@ -28,7 +28,7 @@ struct Workspace {
   size_t stats_off = 0;     // float2 [total_q * Hq][stat_tiles]   per-tile (max, sum-exp2)
   size_t lse_off = 0;       // float  [total_q * Hq]               log2-sum-exp2 per (row, head)
   size_t partial_off = 0;   // float  [Hkv][N]                     per-KV-head score partials
-  size_t logits_off = 0;    // float  [Hq * R][N] (narrow path only; 0 bytes otherwise)
+  size_t logits_off = 0;    // float  [Hq][max_qlen][N] (matrix-vector path only; 0 bytes otherwise)
   // select
   size_t keys_off = 0;      // uint32 [N] (only when a sequence does not fit in shared memory)
   int stat_tiles = 0;
@@ -44,6 +44,13 @@ cudaError_t launch_score(const Shapes& s, const Workspace& w, const void* q, con
 cudaError_t launch_score_generic(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
                                  const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
                                  unsigned char* ws, cudaStream_t stream);
+
+// Few scored rows per sequence (the paper's fine stage scores the last token only): matrix-vector path.
+constexpr int kNarrowMaxRows = 4;
+bool score_narrow_applies(const Shapes& s);
+cudaError_t launch_score_narrow(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
+                                const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
+                                unsigned char* ws, cudaStream_t stream);
 
 cudaError_t launch_select(const Shapes& s, const Workspace& w, const float* scores, const int32_t* cu_seqlens,
                           const int32_t* keep_counts, const uint8_t* protect, const int32_t* q_idx,

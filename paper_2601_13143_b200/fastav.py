@@ -17,6 +17,10 @@ FASTAV_CAUSAL = 1
 FASTAV_PROTECT_QUERY_ROWS = 2
 FASTAV_KEEP_IDX_GLOBAL = 4
 
+FASTAV_SCORE_PATH_GENERIC = 0x100
+FASTAV_SCORE_PATH_NARROW = 0x200
+FASTAV_SCORE_PATH_WIDE = 0x300
+
 FASTAV_DEV_K_CLAMPED = 1
 FASTAV_DEV_PROTECT_OVERFLOW = 2
 FASTAV_DEV_WAIT_EXPIRED = 4

@@ -24,7 +24,7 @@ def flags_of(p) -> int:
     return (fastav.FASTAV_CAUSAL if p.causal else 0) | (fastav.FASTAV_PROTECT_QUERY_ROWS if p.protect_rows else 0)
 
 
-def to_device(p, hidden=None, pos=None, protect=None, flags=None, device="cuda") -> fastav.PruneBuffers:
+def to_device(p, hidden=None, pos=None, protect=None, flags=None, device="cuda", extra_flags=0) -> fastav.PruneBuffers:
     """PruneInputs (CPU) -> device buffers + outputs.  ``hidden``/``pos`` override the problem's own
     (used by chained stages)."""
     hidden = p.hidden if hidden is None else hidden
@@ -35,7 +35,7 @@ def to_device(p, hidden=None, pos=None, protect=None, flags=None, device="cuda")
     return fastav.make_buffers(q=dev(p.q), q_idx=dev(p.q_idx), cu_qlens=dev(p.cu_qlens), k=dev(p.k), v=dev(p.v),
                                cu_seqlens=dev(p.cu_seqlens), keep_counts=dev(p.keep_counts), hidden=dev(hidden), pos=dev(pos),
                                protect=dev(protect), softmax_scale=p.softmax_scale,
-                               flags=flags_of(p) if flags is None else flags, lens=lens, rows=rows, keeps=p.keep_counts.tolist())
+                               flags=(flags_of(p) if flags is None else flags) | extra_flags, lens=lens, rows=rows, keeps=p.keep_counts.tolist())
 
 
 def oracle_scores(p, nthreads=0) -> np.ndarray:

@@ -31,16 +31,33 @@ SCORE_CASES = [
     ([333, 0, 65], [4, 0, 3], 32, 8, 128),
     ([200], [0], 8, 2, 64),
     ([2500], [5], 4, 2, 128),
+    ([3000, 17], [1, 1], 32, 8, 128),
+    ([1111], [2], 12, 3, 64),
+    ([700, 900], [4, 3], 28, 4, 128),
+    ([513], [1], 16, 16, 64),
 ]
+
+
+SCORE_PATHS = {"auto": 0, "generic": fastav.FASTAV_SCORE_PATH_GENERIC, "narrow": fastav.FASTAV_SCORE_PATH_NARROW,
+               "wide": fastav.FASTAV_SCORE_PATH_WIDE}
+
+
+def _path_applies(path, rows, hq, hkv, d):
+    if path == "narrow":
+        return 1 <= max(rows) <= 4
+    return True
 
 
 @pytest.mark.parametrize("lens,rows,hq,hkv,d", SCORE_CASES)
 @pytest.mark.parametrize("causal", [True, False])
-def test_score_matches_oracle(lens, rows, hq, hkv, d, causal):
+@pytest.mark.parametrize("path", ["auto", "generic", "narrow"])
+def test_score_matches_oracle(lens, rows, hq, hkv, d, causal, path):
+    if not _path_applies(path, rows, hq, hkv, d):
+        pytest.skip("path does not take these shapes")
     p = W.random_problem(seed=sum(lens) + hq, lens=lens, rows=rows, keeps=[n // 2 for n in lens], num_q_heads=hq,
                          num_kv_heads=hkv, head_dim=d, hidden=64, duplicate_keys=3, trailing_rows=False)
     p.causal = causal
-    buf = parity.to_device(p)
+    buf = parity.to_device(p, extra_flags=SCORE_PATHS[path])
     buf.scores.fill_(float("nan"))
     buf.score()
     torch.cuda.synchronize()
