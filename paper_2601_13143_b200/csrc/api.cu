@@ -139,7 +139,8 @@ Workspace plan_workspace(const fastav_params& p) {
   w.stat_tiles = (p.max_seqlen + 63) / 64;
   w.stats_off = carve(rows_heads * (size_t)w.stat_tiles * sizeof(float2));
   w.lse_off = carve(rows_heads * sizeof(float));
-  w.partial_off = carve((size_t)p.num_kv_heads * p.total_tokens * sizeof(float));
+  w.partial_off = carve((size_t)p.num_kv_heads * wide_row_chunks(p.max_qlen, p.num_q_heads / p.num_kv_heads) *
+                        p.total_tokens * sizeof(float));
   const bool narrow = p.max_qlen >= 1 && p.max_qlen <= kNarrowMaxRows;
   w.logits_off = carve(narrow ? (size_t)p.num_q_heads * p.max_qlen * p.total_tokens * sizeof(float) : 0);
   w.keys_off = carve((size_t)p.total_tokens * sizeof(uint32_t));
@@ -151,18 +152,25 @@ Workspace plan_workspace(const fastav_params& p) {
 bool score_path_ok(const Shapes& s) {
   const unsigned forced = s.flags & FASTAV_SCORE_PATH_MASK;
   if (forced == FASTAV_SCORE_PATH_NARROW) return score_narrow_applies(s);
-  if (forced == FASTAV_SCORE_PATH_WIDE) return false;
+  if (forced == FASTAV_SCORE_PATH_WIDE) return score_wide_applies(s);
   return true;
 }
 
+// Shape-based choice: few scored rows -> matrix-vector path; otherwise the tensor-core path; the
+// CUDA-core tiles take whatever is left (and whatever the TMA descriptor cannot express).
 cudaError_t launch_score(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
                          const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
-                         unsigned char* ws, cudaStream_t stream) {
+                         unsigned char* ws, int32_t* device_status, cudaStream_t stream) {
   const unsigned forced = s.flags & FASTAV_SCORE_PATH_MASK;
   if (forced == FASTAV_SCORE_PATH_GENERIC) return launch_score_generic(s, w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out, ws, stream);
   if (score_narrow_applies(s) && (forced == 0 || forced == FASTAV_SCORE_PATH_NARROW))
     return launch_score_narrow(s, w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out, ws, stream);
-  if (forced != 0) return cudaErrorNotSupported;
+  if (score_wide_applies(s)) {
+    bool used = false;
+    const cudaError_t e = launch_score_wide(s, w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out, ws, device_status, stream, &used);
+    if (used || e != cudaSuccess) return e;
+    if (forced == FASTAV_SCORE_PATH_WIDE) return cudaErrorNotSupported;
+  }
   return launch_score_generic(s, w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out, ws, stream);
 }
 
@@ -201,7 +209,6 @@ int32_t fastav_workspace_bytes(const fastav_params* params, size_t* out_bytes) {
 int32_t fastav_score(const fastav_params* params, const void* q, const int32_t* q_idx, const int32_t* cu_qlens,
                      const void* k, const int32_t* cu_seqlens, const float* lse_opt, float* scores_out,
                      void* workspace, size_t workspace_bytes, int32_t* device_status, void* stream) {
-  (void)device_status;
   int32_t rc = check_params(params);
   if (rc != FASTAV_OK) return rc;
   if (lse_opt) return FASTAV_ERR_UNSUPPORTED;
@@ -211,7 +218,7 @@ int32_t fastav_score(const fastav_params* params, const void* q, const int32_t* 
   if (!score_path_ok(make_shapes(*params))) return FASTAV_ERR_UNSUPPORTED;
   if (params->total_tokens == 0) return FASTAV_OK;
   const cudaError_t e = launch_score(make_shapes(*params), w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out,
-                                     static_cast<unsigned char*>(workspace), static_cast<cudaStream_t>(stream));
+                                     static_cast<unsigned char*>(workspace), device_status, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? FASTAV_OK : cuda_failed(e);
 }
 
@@ -264,7 +271,7 @@ int32_t fastav_prune(const fastav_params* params, const void* q, const int32_t* 
   unsigned char* ws = static_cast<unsigned char*>(workspace);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e = cudaSuccess;
-  if (params->total_tokens > 0) e = launch_score(s, w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out, ws, st);
+  if (params->total_tokens > 0) e = launch_score(s, w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out, ws, device_status, st);
   if (e == cudaSuccess)
     e = launch_select(s, w, scores_out, cu_seqlens, keep_counts, protect_opt, q_idx, cu_qlens, keep_idx_out, cu_keep_out, ws,
                       device_status, st);

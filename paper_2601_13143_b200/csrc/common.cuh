@@ -27,7 +27,7 @@ struct Workspace {
   // generic / narrow score
   size_t stats_off = 0;     // float2 [total_q * Hq][stat_tiles]   per-tile (max, sum-exp2)
   size_t lse_off = 0;       // float  [total_q * Hq]               log2-sum-exp2 per (row, head)
-  size_t partial_off = 0;   // float  [Hkv][N]                     per-KV-head score partials
+  size_t partial_off = 0;   // float  [Hkv * row chunks][N]        score partials per KV head and chunk of query rows
   size_t logits_off = 0;    // float  [Hq][max_qlen][N] (matrix-vector path only; 0 bytes otherwise)
   // select
   size_t keys_off = 0;      // uint32 [N] (only when a sequence does not fit in shared memory)
@@ -39,7 +39,7 @@ Workspace plan_workspace(const fastav_params& p);
 // ---- launchers (each returns cudaGetLastError() after its launches) -------------------------
 cudaError_t launch_score(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
                          const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
-                         unsigned char* ws, cudaStream_t stream);
+                         unsigned char* ws, int32_t* device_status, cudaStream_t stream);
 
 cudaError_t launch_score_generic(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
                                  const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
@@ -51,6 +51,14 @@ bool score_narrow_applies(const Shapes& s);
 cudaError_t launch_score_narrow(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
                                 const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
                                 unsigned char* ws, cudaStream_t stream);
+
+// Many scored rows per sequence: tensor-core path (tcgen05 + TMA).  `*used` is false when the TMA
+// descriptor for K could not be built; nothing was launched then and the caller takes another path.
+int wide_row_chunks(int max_qlen, int group);
+bool score_wide_applies(const Shapes& s);
+cudaError_t launch_score_wide(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
+                              const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
+                              unsigned char* ws, int32_t* device_status, cudaStream_t stream, bool* used);
 
 cudaError_t launch_select(const Shapes& s, const Workspace& w, const float* scores, const int32_t* cu_seqlens,
                           const int32_t* keep_counts, const uint8_t* protect, const int32_t* q_idx,

@@ -35,6 +35,9 @@ SCORE_CASES = [
     ([1111], [2], 12, 3, 64),
     ([700, 900], [4, 3], 28, 4, 128),
     ([513], [1], 16, 16, 64),
+    ([600], [100], 8, 2, 128),          # 400 query rows per KV head: two row chunks on the tensor-core path
+    ([4100, 130], [40, 64], 28, 4, 128),
+    ([2100], [33], 8, 1, 64),           # 264 rows: a second row chunk with only 8 rows
 ]
 
 
@@ -45,12 +48,14 @@ SCORE_PATHS = {"auto": 0, "generic": fastav.FASTAV_SCORE_PATH_GENERIC, "narrow":
 def _path_applies(path, rows, hq, hkv, d):
     if path == "narrow":
         return 1 <= max(rows) <= 4
+    if path == "wide":
+        return max(rows) >= 1
     return True
 
 
 @pytest.mark.parametrize("lens,rows,hq,hkv,d", SCORE_CASES)
 @pytest.mark.parametrize("causal", [True, False])
-@pytest.mark.parametrize("path", ["auto", "generic", "narrow"])
+@pytest.mark.parametrize("path", ["auto", "generic", "narrow", "wide"])
 def test_score_matches_oracle(lens, rows, hq, hkv, d, causal, path):
     if not _path_applies(path, rows, hq, hkv, d):
         pytest.skip("path does not take these shapes")
