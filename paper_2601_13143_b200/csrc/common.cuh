@@ -54,6 +54,7 @@ cudaError_t launch_score_narrow(const Shapes& s, const Workspace& w, const void*
 
 // Many scored rows per sequence: tensor-core path (tcgen05 + TMA).  `*used` is false when the TMA
 // descriptor for K could not be built; nothing was launched then and the caller takes another path.
+int wide_rows_per_chunk(int group);
 int wide_row_chunks(int max_qlen, int group);
 bool score_wide_applies(const Shapes& s);
 cudaError_t launch_score_wide(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,

@@ -27,6 +27,10 @@
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
+#ifndef FASTAV_EPI_SCALAR
+#define FASTAV_EPI_SCALAR 0
+#endif
+
 namespace fastav {
 namespace {
 
@@ -34,9 +38,9 @@ constexpr int kTileKeys = 128;    // keys per K tile
 constexpr int kRowsPerCta = 256;  // query rows (flat over scored row x head of the KV group) per block
 constexpr int kStages = 4;        // K tiles in flight
 constexpr int kThreads = 320;     // warp 0: TMA, warp 1: MMA, warps 2-9: softmax
-constexpr int kEpiThreads = 256;
 constexpr int kTmemCols = 512;
-constexpr int kMaxChunkTiles = 16;
+constexpr int kMaxUnits = 48;       // work units one block may be given (the host sizes key chunks accordingly)
+constexpr int kCtrlBytes = 20 * 1024;
 
 template <int DIM>
 struct Layout {
@@ -48,21 +52,8 @@ struct Layout {
   static constexpr int kQOff = 0;
   static constexpr int kKOff = kQOff + kQBytes;
   static constexpr int kCtrlOff = kKOff + kStages * kKTileBytes;  // barriers and small arrays
-  static constexpr int kTotal = kCtrlOff + 4096 + 1024;           // + slack to align the base to 1024 bytes
+  static constexpr int kTotal = kCtrlOff + kCtrlBytes + 1024;     // + slack to align the base to 1024 bytes
 };
-
-struct Control {
-  uint64_t full_k[kStages], empty_k[kStages];
-  uint64_t q_ready;
-  uint64_t tmem_full[4], tmem_empty[4];
-  uint32_t tmem_base;
-  int abort;
-  int min_limit;
-  int pad;
-  alignas(16) float neg_lse[kRowsPerCta];  // sweep 2: -lse of each query-row column (-inf for padding)
-  alignas(16) int limit[kRowsPerCta];      // sweep 2: last key each column's row may see
-};
-static_assert(sizeof(Control) <= 4096, "control block must fit its slot");
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
@@ -81,108 +72,261 @@ __device__ __forceinline__ void tmem_ld_wait_for(uint32_t (&v)[32]) {
                : "memory");
 }
 
-__device__ __forceinline__ void epilogue_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-
-// Sweep 1, one 32-key piece of a row: fold it into the row's running (max, sum).  Columns above
-// `bound` (relative to the piece's first column) are hidden from this row.
+// Sweep 1, one 32-key piece of a row: fold it into the row's running (max, sum).  Under MASKED,
+// columns above `bound` (relative to the piece's first column) are hidden from this row.  Branch-free:
+// a row that has seen nothing yet carries zmax = -inf and sum 0, and stays that way until a key shows up.
+template <bool MASKED>
 __device__ __forceinline__ void fold_row_piece(const uint32_t (&v)[32], int bound, float scale, float& zmax, float2& sum2) {
-  if (bound < 0) return;
   float z[32];
-  if (bound >= 31) {
 #pragma unroll
-    for (int j = 0; j < 32; ++j) z[j] = __uint_as_float(v[j]);
-  } else {
+  for (int j = 0; j < 32; ++j) z[j] = (!MASKED || j <= bound) ? __uint_as_float(v[j]) : -INFINITY;
+  float m0 = max3(z[0], z[1], z[2]), m1 = max3(z[3], z[4], z[5]);
 #pragma unroll
-    for (int j = 0; j < 32; ++j) z[j] = j <= bound ? __uint_as_float(v[j]) : -INFINITY;
+  for (int j = 6; j + 3 < 32; j += 4) {
+    m0 = max3(m0, z[j], z[j + 1]);
+    m1 = max3(m1, z[j + 2], z[j + 3]);
   }
-  float m = max3(z[0], z[1], z[2]);
+  const float newmax = fmaxf(zmax, max3(m0, m1, fmaxf(z[30], z[31])));
+  const float ref = newmax == -INFINITY ? 0.f : newmax;      // keeps the differences below free of inf - inf
+  const float corr = ptx::ex2_approx((zmax - ref) * scale);  // 1 when the maximum did not move, 0 on the first keys
+  sum2.x *= corr;
+  sum2.y *= corr;
+  zmax = newmax;
+  const float shift = -ref * scale;
+#if FASTAV_EPI_SCALAR
 #pragma unroll
-  for (int j = 3; j + 1 < 32; j += 2) m = max3(m, z[j], z[j + 1]);
-  m = fmaxf(m, z[31]);
-  const float newmax = fmaxf(zmax, m);
-  if (newmax == -INFINITY) return;  // nothing visible so far
-  if (newmax != zmax) {             // rescale what has been summed under the old maximum
-    const float corr = ptx::ex2_approx((zmax - newmax) * scale);
-    sum2.x *= corr;
-    sum2.y *= corr;
-    zmax = newmax;
+  for (int j = 0; j < 32; j += 2) {
+    sum2.x += ptx::ex2_approx(fmaf(z[j], scale, shift));
+    sum2.y += ptx::ex2_approx(fmaf(z[j + 1], scale, shift));
   }
-  const float shift = -newmax * scale;
+#else
   const float2 sc = make_float2(scale, scale), sh = make_float2(shift, shift);
 #pragma unroll
   for (int j = 0; j < 32; j += 2) {
     const float2 x = __ffma2_rn(make_float2(z[j], z[j + 1]), sc, sh);
     sum2 = __fadd2_rn(sum2, make_float2(ptx::ex2_approx(x.x), ptx::ex2_approx(x.y)));
   }
+#endif
+}
+
+__device__ __forceinline__ void fold_row_piece_any(const uint32_t (&v)[32], int bound, float scale, float& zmax, float2& sum2) {
+  if (bound >= 31) fold_row_piece<false>(v, bound, scale, zmax, sum2);
+  else fold_row_piece<true>(v, bound, scale, zmax, sum2);
+  __syncwarp();  // rows of one warp may differ in `bound`; the tcgen05 instructions that follow need the whole warp
 }
 
 // Sweep 2, 32 query-row columns of one key: add 2^(z - lse).  `key` is the sequence-local key index;
-// under `masked`, a column whose row may not see the key adds nothing.
-__device__ __forceinline__ void add_key_piece(const uint32_t (&v)[32], const float* neg_lse, const int* limit, bool masked,
-                                              int key, float scale, float2& sum2) {
-  const float2 sc = make_float2(scale, scale);
+// under MASKED, a column whose row may not see the key adds nothing.
+template <bool MASKED>
+__device__ __forceinline__ void add_key_piece(const uint32_t (&v)[32], const float* neg_lse, const int* limit, int key,
+                                              float scale, float2& sum2) {
 #pragma unroll
   for (int j = 0; j < 32; j += 4) {
     const float4 nl = *reinterpret_cast<const float4*>(neg_lse + j);
+#if FASTAV_EPI_SCALAR
+    float p0 = ptx::ex2_approx(fmaf(__uint_as_float(v[j]), scale, nl.x));
+    float p1 = ptx::ex2_approx(fmaf(__uint_as_float(v[j + 1]), scale, nl.y));
+    float p2 = ptx::ex2_approx(fmaf(__uint_as_float(v[j + 2]), scale, nl.z));
+    float p3 = ptx::ex2_approx(fmaf(__uint_as_float(v[j + 3]), scale, nl.w));
+#else
+    const float2 sc = make_float2(scale, scale);
     const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(v[j]), __uint_as_float(v[j + 1])), sc, make_float2(nl.x, nl.y));
     const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])), sc, make_float2(nl.z, nl.w));
     float p0 = ptx::ex2_approx(x0.x), p1 = ptx::ex2_approx(x0.y), p2 = ptx::ex2_approx(x1.x), p3 = ptx::ex2_approx(x1.y);
-    if (masked) {
+#endif
+    if (MASKED) {
       const int4 lim = *reinterpret_cast<const int4*>(limit + j);
       p0 = key <= lim.x ? p0 : 0.f;
       p1 = key <= lim.y ? p1 : 0.f;
       p2 = key <= lim.z ? p2 : 0.f;
       p3 = key <= lim.w ? p3 : 0.f;
     }
+#if FASTAV_EPI_SCALAR
+    sum2.x += p0; sum2.y += p1; sum2.x += p2; sum2.y += p3;
+#else
     sum2 = __fadd2_rn(sum2, make_float2(p0, p1));
     sum2 = __fadd2_rn(sum2, make_float2(p2, p3));
+#endif
   }
+}
+
+// Sweep 2, all query-row columns of one key: the accumulator is read 32 columns at a time, the next
+// read in flight while the current one is summed.
+template <bool MASKED>
+__device__ __forceinline__ float sum_key_columns(uint32_t taddr, int pieces, const float* neg_lse, const int* limit, int key,
+                                                 float scale) {
+  float2 sum2 = make_float2(0.f, 0.f);
+  uint32_t va[32], vb[32];
+  ptx::tmem_ld32(taddr, va);
+  int c = 0;
+#pragma unroll 1
+  for (; c + 2 <= pieces; c += 2) {
+    tmem_ld_wait_for(va);
+    ptx::tmem_ld32(taddr + (c + 1) * 32, vb);
+    add_key_piece<MASKED>(va, neg_lse + c * 32, limit + c * 32, key, scale, sum2);
+    tmem_ld_wait_for(vb);
+    if (c + 2 < pieces) ptx::tmem_ld32(taddr + (c + 2) * 32, va);
+    add_key_piece<MASKED>(vb, neg_lse + (c + 1) * 32, limit + (c + 1) * 32, key, scale, sum2);
+  }
+  if (c < pieces) {
+    tmem_ld_wait_for(va);
+    add_key_piece<MASKED>(va, neg_lse + c * 32, limit + c * 32, key, scale, sum2);
+  }
+  return sum2.x + sum2.y;
+}
+
+// What one block works on at a time: a run of K tiles of one (sequence, KV head, chunk of query rows).
+struct Unit {
+  int tok0, n;         // the sequence: first token in the packed batch, length
+  int row0;            // first scored row of the sequence in q / q_idx
+  int g, rc, kc;       // KV head, query-row chunk, key chunk
+  int rows_here;       // query rows of the chunk that exist (a multiple of G)
+  int new_q;           // the query tile differs from the previous unit's
+};
+
+struct Control {
+  uint64_t full_k[kStages], empty_k[kStages];
+  uint64_t q_ready, q_free;
+  uint64_t tmem_full[4], tmem_empty[4];
+  uint32_t tmem_base;
+  int abort;
+  int n_units;
+  int start_b, start_off;
+  int warp_sums[kThreads / 32];
+  alignas(16) float neg_lse[8][kRowsPerCta];  // sweep 2, per softmax warp: -lse of each query-row column (-inf: padding)
+  alignas(16) int limit[8][kRowsPerCta];      // sweep 2, per softmax warp: last key each column's row may see
+  Unit units[kMaxUnits];
+};
+static_assert(sizeof(Control) <= kCtrlBytes, "control block must fit its slot");
+
+// Number of work units of sequence b: KV heads x query-row chunks x key chunks (0 for an empty sequence
+// or one without scored rows).
+__device__ __forceinline__ int units_of_sequence(const Shapes& s, const int32_t* cu_seqlens, const int32_t* cu_qlens, int b,
+                                                 int rows_per_chunk, int chunk_keys) {
+  const int n = cu_seqlens[b + 1] - cu_seqlens[b];
+  const int flat_rows = (cu_qlens[b + 1] - cu_qlens[b]) * s.group;
+  if (n <= 0 || flat_rows <= 0) return 0;
+  return s.hkv * ((flat_rows + rows_per_chunk - 1) / rows_per_chunk) * ((n + chunk_keys - 1) / chunk_keys);
+}
+
+// Block-wide sum of one int per thread (all threads get the result).
+__device__ __forceinline__ int block_sum(int v, int* warp_sums) {
+#pragma unroll
+  for (int d = 16; d; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = v;
+  __syncthreads();
+  int total = 0;
+#pragma unroll
+  for (int w = 0; w < kThreads / 32; ++w) total += warp_sums[w];
+  return total;
 }
 
 template <int DIM, int SWEEP>
 __global__ void __launch_bounds__(kThreads, 1)
-score_wide_kernel(const __grid_constant__ CUtensorMap k_map, Shapes s, const uint16_t* __restrict__ q,
+score_wide_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap q_map, Shapes s,
                   const int32_t* __restrict__ q_idx, const int32_t* __restrict__ cu_qlens,
-                  const int32_t* __restrict__ cu_seqlens, int chunk_tiles, int stat_chunks, int rc_max,
+                  const int32_t* __restrict__ cu_seqlens, int chunk_tiles, int stat_chunks, int rc_max, int rows_per_chunk,
                   float2* __restrict__ stats, const float* __restrict__ lse, float* __restrict__ partial,
                   int32_t* device_status) {
   using L = Layout<DIM>;
   extern __shared__ unsigned char smem_raw[];
-
-  // ---- which piece of work is this block? (uniform per block; empty pieces leave before any set-up)
-  const int b = blockIdx.z, g = blockIdx.y / rc_max, rc = blockIdx.y % rc_max, kc = blockIdx.x;
-  const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
-  const int row0 = cu_qlens[b], flat_rows = (cu_qlens[b + 1] - row0) * s.group;
-  const int key_begin = kc * chunk_tiles * kTileKeys;
-  if (key_begin >= n || rc * kRowsPerCta >= flat_rows) return;
-  const int rows_here = min(kRowsPerCta, flat_rows - rc * kRowsPerCta);
-  const int tiles = (min(n - key_begin, chunk_tiles * kTileKeys) + kTileKeys - 1) / kTileKeys;
-  const int mtiles = (rows_here + 127) / 128;         // sweep 1: 128-row MMA tiles in use
-  const int n_cols = (rows_here + 31) / 32 * 32;      // sweep 2: MMA N (query rows as columns)
-  const bool causal = (s.flags & FASTAV_CAUSAL) != 0;
-
   const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_raw + (base - ptx::smem_u32(smem_raw));
   Control& ctl = *reinterpret_cast<Control*>(base_ptr + L::kCtrlOff);
   const uint32_t q_smem = base + L::kQOff, k_smem = base + L::kKOff;
   volatile int* abort = &ctl.abort;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int chunk_keys = chunk_tiles * kTileKeys;
+  const bool causal = (s.flags & FASTAV_CAUSAL) != 0;
+  const int scored_per_chunk = rows_per_chunk / s.group;  // scored rows per query-row chunk (a multiple of 8)
 
+  // ---- this block's share of the work: units [u0, u1) of the list ordered by (sequence, KV head,
+  //      row chunk, key chunk), so that consecutive units mostly share their query tile -------------
+  int total_units = 0;
+  for (int b0 = 0; b0 < s.batch; b0 += kThreads) {
+    const int b = b0 + threadIdx.x;
+    total_units += block_sum(b < s.batch ? units_of_sequence(s, cu_seqlens, cu_qlens, b, rows_per_chunk, chunk_keys) : 0,
+                             ctl.warp_sums);
+  }
+  const int u0 = (int)((long long)total_units * blockIdx.x / gridDim.x);
+  const int u1 = (int)((long long)total_units * (blockIdx.x + 1) / gridDim.x);
+  if (u1 <= u0) return;  // uniform: nothing for this block
+  {
+    int before = 0;  // units of the sequences before the current batch slice
+    for (int b0 = 0; b0 < s.batch; b0 += kThreads) {
+      const int b = b0 + threadIdx.x;
+      const int mine = b < s.batch ? units_of_sequence(s, cu_seqlens, cu_qlens, b, rows_per_chunk, chunk_keys) : 0;
+      int incl = mine;  // inclusive scan inside the warp, then across warps through shared memory
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int t = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+        if (lane >= d) incl += t;
+      }
+      __syncthreads();
+      if (lane == 31) ctl.warp_sums[warp] = incl;
+      __syncthreads();
+      int warp_base = 0, slice_total = 0;
+#pragma unroll
+      for (int w = 0; w < kThreads / 32; ++w) {
+        if (w < warp) warp_base += ctl.warp_sums[w];
+        slice_total += ctl.warp_sums[w];
+      }
+      const int excl = before + warp_base + incl - mine;
+      if (mine > 0 && excl <= u0 && u0 < excl + mine) {  // exactly one thread of one slice
+        ctl.start_b = b;
+        ctl.start_off = u0 - excl;
+      }
+      before += slice_total;
+    }
+  }
+  __syncthreads();
   if (threadIdx.x == 0) {
+    // Walk the units of this block and write them down for every role.
+    int b = ctl.start_b, off = ctl.start_off, count = 0, prev_b = -1, prev_grc = -1;
+    for (int u = u0; u < u1 && count < kMaxUnits; ++u) {
+      int tok0, n, row0, flat_rows, row_chunks, key_chunks;
+      for (;;) {
+        tok0 = cu_seqlens[b];
+        n = cu_seqlens[b + 1] - tok0;
+        row0 = cu_qlens[b];
+        flat_rows = (cu_qlens[b + 1] - row0) * s.group;
+        row_chunks = (flat_rows + rows_per_chunk - 1) / rows_per_chunk;
+        key_chunks = (n + chunk_keys - 1) / chunk_keys;
+        if (n > 0 && flat_rows > 0 && off < s.hkv * row_chunks * key_chunks) break;
+        ++b;  // sequence exhausted (or empty): on to the next one
+        off = 0;
+      }
+      const int grc = off / key_chunks;
+      Unit un;
+      un.tok0 = tok0; un.n = n; un.row0 = row0;
+      un.g = grc / row_chunks; un.rc = grc % row_chunks; un.kc = off % key_chunks;
+      un.rows_here = min(rows_per_chunk, flat_rows - un.rc * rows_per_chunk);
+      un.new_q = (b != prev_b || grc != prev_grc) ? 1 : 0;
+      prev_b = b; prev_grc = grc;
+      ctl.units[count++] = un;
+      ++off;
+    }
+    ctl.n_units = count;
     for (int i = 0; i < kStages; ++i) {
       ptx::mbar_init(ptx::smem_u32(&ctl.full_k[i]), 1);
       ptx::mbar_init(ptx::smem_u32(&ctl.empty_k[i]), 1);
     }
-    ptx::mbar_init(ptx::smem_u32(&ctl.q_ready), kEpiThreads);
+    ptx::mbar_init(ptx::smem_u32(&ctl.q_ready), 1);
+    ptx::mbar_init(ptx::smem_u32(&ctl.q_free), 1);
     for (int i = 0; i < 4; ++i) {
       ptx::mbar_init(ptx::smem_u32(&ctl.tmem_full[i]), 1);
       ptx::mbar_init(ptx::smem_u32(&ctl.tmem_empty[i]), 128);
     }
     ctl.abort = 0;
-    ctl.min_limit = INT_MAX;
     ptx::fence_barrier_init();
     ptx::prefetch_tensormap(&k_map);
+    ptx::prefetch_tensormap(&q_map);
   }
+  // The query tile starts as zeros: rows no copy ever fills are then harmless operands.
+  for (int i = threadIdx.x; i < L::kQBytes / 16; i += kThreads)
+    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(q_smem + i * 16), "r"(0) : "memory");
+  ptx::fence_proxy_async_smem();  // ordered before the TMA writes that follow the barrier
   if (warp == 1) {
     ptx::tmem_alloc(ptx::smem_u32(&ctl.tmem_base), kTmemCols);
     ptx::tmem_relinquish();
@@ -191,184 +335,222 @@ score_wide_kernel(const __grid_constant__ CUtensorMap k_map, Shapes s, const uin
   __syncthreads();
   ptx::tc_fence_after_sync();
   const uint32_t tmem = ctl.tmem_base;
+  const int n_units = ctl.n_units;
 
   if (warp == 0) {
-    // ---- TMA producer: one elected lane streams the K tiles of this block's key chunk ----------
+    // ---- TMA producer: one elected lane streams query tiles and K tiles ---------------------------
     if (lane == 0) {
-      int issued = 0;
-      for (int t = 0; t < tiles; ++t) {
-        const int stage = t % kStages;
-        const uint32_t parity = (t / kStages) & 1;
-        if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.empty_k[stage]), parity ^ 1u, abort)) break;
-        const uint32_t bar = ptx::smem_u32(&ctl.full_k[stage]);
-        ptx::mbar_arrive_expect_tx(bar, L::kKTileBytes);
+      int tile_no = 0, q_gen = 0;  // K tiles / query tiles issued so far
+      bool ok = true;
+      for (int u = 0; u < n_units && ok; ++u) {
+        const Unit un = ctl.units[u];
+        if (un.new_q) {
+          // The previous query tile must have been read by its last MMA before it is overwritten.
+          if (q_gen > 0) ok = ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.q_free), (q_gen - 1) & 1, abort);
+          if (!ok) break;
+          // Boxes of 8 scored rows x G heads x 64 columns land as 8 G consecutive 128-byte rows, which is the
+          // flat (scored row, head) order of the tile; 8 G rows are a whole number of 1024-byte swizzle groups.
+          const int boxes = (un.rows_here / s.group + 7) / 8;
+          const uint32_t box_bytes = 8u * s.group * 128u;
+          const uint32_t bar = ptx::smem_u32(&ctl.q_ready);
+          ptx::mbar_arrive_expect_tx(bar, boxes * box_bytes * L::kSubTiles);
+          for (int sub = 0; sub < L::kSubTiles; ++sub)
+            for (int i = 0; i < boxes; ++i)
+              ptx::tma_load_3d(q_smem + sub * L::kQSubBytes + i * box_bytes, &q_map, sub * 64, un.g * s.group,
+                               un.row0 + un.rc * scored_per_chunk + 8 * i, bar);
+          ++q_gen;
+        }
+        const int key_begin = un.kc * chunk_keys;
+        const int tiles = (min(un.n - key_begin, chunk_keys) + kTileKeys - 1) / kTileKeys;
+        for (int t = 0; t < tiles; ++t, ++tile_no) {
+          const int stage = tile_no % kStages;
+          ok = ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.empty_k[stage]), ((tile_no / kStages) & 1) ^ 1u, abort);
+          if (!ok) break;
+          const uint32_t bar = ptx::smem_u32(&ctl.full_k[stage]);
+          ptx::mbar_arrive_expect_tx(bar, L::kKTileBytes);
 #pragma unroll
-        for (int sub = 0; sub < L::kSubTiles; ++sub)
-          ptx::tma_load_3d(k_smem + stage * L::kKTileBytes + sub * L::kKSubBytes, &k_map, sub * 64, g,
-                           tok0 + key_begin + t * kTileKeys, bar);
-        issued = t + 1;
+          for (int sub = 0; sub < L::kSubTiles; ++sub)
+            ptx::tma_load_3d(k_smem + stage * L::kKTileBytes + sub * L::kKSubBytes, &k_map, sub * 64, un.g,
+                             un.tok0 + key_begin + t * kTileKeys, bar);
+        }
       }
       if (*abort) {
-        // Giving up: the copies already issued still write into this block's shared memory, so wait
-        // (bounded once more) for each of them before the block may exit.
+        // Giving up: copies already issued still write into this block's shared memory, so wait (bounded
+        // once more) for each of them before the block may exit.
         int never = 0;
-        for (int t = max(0, issued - kStages); t < issued; ++t)
+        for (int t = max(0, tile_no - kStages); t < tile_no; ++t)
           ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.full_k[t % kStages]), (t / kStages) & 1, &never);
+        if (q_gen > 0) ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.q_ready), (q_gen - 1) & 1, &never);
       }
     }
   } else if (warp == 1) {
-    // ---- MMA issuer: one elected lane ----------------------------------------------------------
-    if (lane == 0 && ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.q_ready), 0, abort)) {
-      ptx::tc_fence_after_sync();
-      for (int t = 0; t < tiles; ++t) {
-        const int stage = t % kStages, buf = t & 1;
-        const uint32_t parity = (t / kStages) & 1, buf_parity = (t >> 1) & 1;
-        if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.full_k[stage]), parity, abort)) break;
-        const uint32_t k_tile = k_smem + stage * L::kKTileBytes;
-        if constexpr (SWEEP == 1) {
-          // S = Q K^T: A = 128 query rows, B = 128 keys; accumulator (buf, e) at columns buf*256 + e*128.
-          bool ok = true;
-          for (int e = 0; e < mtiles && ok; ++e) {
-            ok = ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.tmem_empty[buf * 2 + e]), buf_parity ^ 1u, abort);
+    // ---- MMA issuer: one elected lane -------------------------------------------------------------
+    if (lane == 0) {
+      int tile_no = 0, q_gen = 0;
+      int uses0 = 0, uses1 = 0;  // sweep 1: how often the accumulators of 128-row tile e have been used
+      bool ok = true;
+      for (int u = 0; u < n_units && ok; ++u) {
+        const Unit un = ctl.units[u];
+        if (un.new_q) {
+          ok = ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.q_ready), q_gen & 1, abort);
+          if (!ok) break;
+          ptx::tc_fence_after_sync();
+          ++q_gen;
+        }
+        const int key_begin = un.kc * chunk_keys;
+        const int tiles = (min(un.n - key_begin, chunk_keys) + kTileKeys - 1) / kTileKeys;
+        const int mtiles = (un.rows_here + 127) / 128;     // sweep 1: 128-row MMA tiles in use
+        const int n_cols = (un.rows_here + 31) / 32 * 32;  // sweep 2: MMA N (query rows as columns)
+        for (int t = 0; t < tiles && ok; ++t, ++tile_no) {
+          const int stage = tile_no % kStages;
+          ok = ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.full_k[stage]), (tile_no / kStages) & 1, abort);
+          if (!ok) break;
+          const uint32_t k_tile = k_smem + stage * L::kKTileBytes;
+          if constexpr (SWEEP == 1) {
+            // S = Q K^T: A = 128 query rows, B = 128 keys; accumulator (e, i) at columns i*256 + e*128.
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              if (e >= mtiles || !ok) break;
+              const int uses = e == 0 ? uses0 : uses1;
+              const int i = uses & 1;
+              ok = ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.tmem_empty[i * 2 + e]), ((uses >> 1) & 1) ^ 1u, abort);
+              if (!ok) break;
+              ptx::tc_fence_after_sync();
+#pragma unroll
+              for (int ks = 0; ks < DIM / 16; ++ks) {
+                const uint32_t sub = ks / 4, off = (ks % 4) * 32;
+                ptx::umma_bf16(tmem + i * 256 + e * 128, ptx::umma_desc_sw128(q_smem + sub * L::kQSubBytes + e * 128 * 128, off),
+                               ptx::umma_desc_sw128(k_tile + sub * L::kKSubBytes, off), ptx::umma_idesc_bf16(128, kTileKeys),
+                               ks > 0);
+              }
+              ptx::umma_commit(ptx::smem_u32(&ctl.tmem_full[i * 2 + e]));
+              if (e == 0) ++uses0; else ++uses1;
+            }
+            if (!ok) break;
+            ptx::umma_commit(ptx::smem_u32(&ctl.empty_k[stage]));
+          } else {
+            // S^T = K Q^T: A = 128 keys, B = n_cols query rows; accumulator i at columns i*256.
+            const int i = tile_no & 1;
+            ok = ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.tmem_empty[i]), ((tile_no >> 1) & 1) ^ 1u, abort);
             if (!ok) break;
             ptx::tc_fence_after_sync();
+            const uint32_t idesc = ptx::umma_idesc_bf16(kTileKeys, n_cols);
 #pragma unroll
             for (int ks = 0; ks < DIM / 16; ++ks) {
               const uint32_t sub = ks / 4, off = (ks % 4) * 32;
-              ptx::umma_bf16(tmem + buf * 256 + e * 128, ptx::umma_desc_sw128(q_smem + sub * L::kQSubBytes + e * 128 * 128, off),
-                             ptx::umma_desc_sw128(k_tile + sub * L::kKSubBytes, off), ptx::umma_idesc_bf16(128, kTileKeys),
-                             ks > 0);
+              ptx::umma_bf16(tmem + i * 256, ptx::umma_desc_sw128(k_tile + sub * L::kKSubBytes, off),
+                             ptx::umma_desc_sw128(q_smem + sub * L::kQSubBytes, off), idesc, ks > 0);
             }
-            ptx::umma_commit(ptx::smem_u32(&ctl.tmem_full[buf * 2 + e]));
+            ptx::umma_commit(ptx::smem_u32(&ctl.empty_k[stage]));
+            ptx::umma_commit(ptx::smem_u32(&ctl.tmem_full[i]));
           }
-          if (!ok) break;
-          ptx::umma_commit(ptx::smem_u32(&ctl.empty_k[stage]));
-        } else {
-          // S^T = K Q^T: A = 128 keys, B = n_cols query rows; accumulator buf at columns buf*256.
-          if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.tmem_empty[buf]), buf_parity ^ 1u, abort)) break;
-          ptx::tc_fence_after_sync();
-          const uint32_t idesc = ptx::umma_idesc_bf16(kTileKeys, n_cols);
-#pragma unroll
-          for (int ks = 0; ks < DIM / 16; ++ks) {
-            const uint32_t sub = ks / 4, off = (ks % 4) * 32;
-            ptx::umma_bf16(tmem + buf * 256, ptx::umma_desc_sw128(k_tile + sub * L::kKSubBytes, off),
-                           ptx::umma_desc_sw128(q_smem + sub * L::kQSubBytes, off), idesc, ks > 0);
-          }
-          ptx::umma_commit(ptx::smem_u32(&ctl.empty_k[stage]));
-          ptx::umma_commit(ptx::smem_u32(&ctl.tmem_full[buf]));
         }
+        // Once the MMAs issued so far are done, the query tile may be replaced.
+        if (ok && u + 1 < n_units && ctl.units[u + 1].new_q) ptx::umma_commit(ptx::smem_u32(&ctl.q_free));
       }
     }
   } else {
     // ---- softmax warps ---------------------------------------------------------------------------
-    const int et = threadIdx.x - 64;          // 0..255
     const int wg = (warp - 2) >> 2;           // warpgroup 0 / 1
     const int quarter = warp & 3;             // the 32 TMEM lanes this warp may read
     const int my_lane = quarter * 32 + lane;  // row (sweep 1) or key (sweep 2) inside the tile
-    const long long q_row_base = (long long)row0 * s.q_st + (long long)g * s.group * s.q_sh;
-
-    // Query tile -> shared memory, in the 128-byte-swizzled K-major layout the MMA descriptors describe.
-    // Flat row f of the KV group is (scored row f / G, head f % G); rows past the end are zero.
-    constexpr int kPieces = DIM / 8;  // 16-byte pieces per row
-    for (int idx = et; idx < kRowsPerCta * kPieces; idx += kEpiThreads) {
-      const int row = idx / kPieces, piece = idx % kPieces;
-      uint4 val = make_uint4(0, 0, 0, 0);
-      if (row < rows_here) {
-        const int f = rc * kRowsPerCta + row;
-        val = __ldg(reinterpret_cast<const uint4*>(q + q_row_base + (long long)(f / s.group) * s.q_st +
-                                                   (long long)(f % s.group) * s.q_sh + piece * 8));
-      }
-      const uint32_t dst = q_smem + (piece / 8) * L::kQSubBytes + row * 128 + (((piece % 8) ^ (row & 7)) << 4);
-      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(val.x), "r"(val.y), "r"(val.z), "r"(val.w) : "memory");
-    }
-    if constexpr (SWEEP == 2) {
-      // Per column (query row): -lse and the last key the row may see.
-      const int f = rc * kRowsPerCta + et;
-      float nl = -INFINITY;
-      int lim = -1;
-      if (et < rows_here) {
-        const int r = f / s.group;
-        nl = -lse[(long long)(row0 + r) * s.hq + g * s.group + f % s.group];
-        lim = causal ? q_idx[row0 + r] : INT_MAX;
-        atomicMin(&ctl.min_limit, lim);
-      }
-      ctl.neg_lse[et] = nl;
-      ctl.limit[et] = lim;
-    }
-    ptx::fence_proxy_async_smem();  // the MMA reads the tile through the async proxy
-    ptx::mbar_arrive(ptx::smem_u32(&ctl.q_ready));
-    epilogue_barrier();
-
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
+
     if constexpr (SWEEP == 1) {
       // Warpgroup e owns the rows of 128-row tile e: thread <-> row.
       const int e = wg;
-      const int f = rc * kRowsPerCta + e * 128 + my_lane;
-      const bool row_valid = e * 128 + my_lane < rows_here;
-      const int r = row_valid ? f / s.group : 0;
-      const int last_visible = min(n - 1, (causal && row_valid) ? q_idx[row0 + r] : INT_MAX);
-      float zmax = -INFINITY;
-      float2 sum2 = make_float2(0.f, 0.f);
-      if (e < mtiles) {
-        for (int t = 0; t < tiles; ++t) {
-          const int buf = t & 1;
-          if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.tmem_full[buf * 2 + e]), (t >> 1) & 1, abort)) break;
+      int uses = 0;
+      bool ok = true;
+      for (int u = 0; u < n_units && ok; ++u) {
+        const Unit un = ctl.units[u];
+        if (e * 128 >= un.rows_here) continue;  // this 128-row tile is not in use for the unit
+        const int key_begin = un.kc * chunk_keys;
+        const int tiles = (min(un.n - key_begin, chunk_keys) + kTileKeys - 1) / kTileKeys;
+        const int f = un.rc * rows_per_chunk + e * 128 + my_lane;
+        const bool row_valid = e * 128 + my_lane < un.rows_here;
+        const int r = row_valid ? f / s.group : 0;
+        const int last_visible = min(un.n - 1, (causal && row_valid) ? q_idx[un.row0 + r] : INT_MAX);
+        float zmax = -INFINITY;
+        float2 sum2 = make_float2(0.f, 0.f);
+        for (int t = 0; t < tiles; ++t, ++uses) {
+          const int i = uses & 1;
+          ok = ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.tmem_full[i * 2 + e]), (uses >> 1) & 1, abort);
+          if (!ok) break;
           ptx::tc_fence_after_sync();
           const int bound = last_visible - (key_begin + t * kTileKeys);  // columns 0..bound of this tile are visible
-          const uint32_t taddr = lane_addr + buf * 256 + e * 128;
+          const uint32_t taddr = lane_addr + i * 256 + e * 128;
           uint32_t va[32], vb[32];
           ptx::tmem_ld32(taddr, va);
           tmem_ld_wait_for(va);
           ptx::tmem_ld32(taddr + 32, vb);
-          fold_row_piece(va, bound, s.scale_log2, zmax, sum2);
-          __syncwarp();  // the rows of a warp may have taken different branches; tcgen05.ld needs them together
+          fold_row_piece_any(va, bound, s.scale_log2, zmax, sum2);
           tmem_ld_wait_for(vb);
           ptx::tmem_ld32(taddr + 64, va);
-          fold_row_piece(vb, bound - 32, s.scale_log2, zmax, sum2);
-          __syncwarp();
+          fold_row_piece_any(vb, bound - 32, s.scale_log2, zmax, sum2);
           tmem_ld_wait_for(va);
           ptx::tmem_ld32(taddr + 96, vb);
-          fold_row_piece(va, bound - 64, s.scale_log2, zmax, sum2);
-          __syncwarp();
+          fold_row_piece_any(va, bound - 64, s.scale_log2, zmax, sum2);
           tmem_ld_wait_for(vb);
           ptx::tc_fence_before_sync();
-          ptx::mbar_arrive(ptx::smem_u32(&ctl.tmem_empty[buf * 2 + e]));  // the accumulator may be overwritten
-          fold_row_piece(vb, bound - 96, s.scale_log2, zmax, sum2);
-          __syncwarp();
+          ptx::mbar_arrive(ptx::smem_u32(&ctl.tmem_empty[i * 2 + e]));  // the accumulator may be overwritten
+          fold_row_piece_any(vb, bound - 96, s.scale_log2, zmax, sum2);
         }
-        if (row_valid) {
-          const long long rh = (long long)(row0 + r) * s.hq + g * s.group + f % s.group;
-          stats[rh * stat_chunks + kc] = make_float2(zmax * s.scale_log2, sum2.x + sum2.y);
+        if (ok && row_valid) {
+          const long long rh = (long long)(un.row0 + r) * s.hq + un.g * s.group + f % s.group;
+          stats[rh * stat_chunks + un.kc] = make_float2(zmax * s.scale_log2, sum2.x + sum2.y);
         }
       }
     } else {
-      // Warpgroup w owns the K tiles of parity w: thread <-> key, all query-row columns.
-      float* out = partial + (long long)(g * rc_max + rc) * s.total_tokens + tok0;
-      const int pieces = n_cols / 32;
-      for (int t = wg; t < tiles; t += 2) {
-        const int buf = t & 1;  // == wg
-        if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.tmem_full[buf]), (t >> 1) & 1, abort)) break;
-        ptx::tc_fence_after_sync();
-        const int key = key_begin + t * kTileKeys + my_lane;
-        const bool masked = causal && (key_begin + t * kTileKeys + kTileKeys - 1 > ctl.min_limit);
-        const uint32_t taddr = lane_addr + buf * 256;
-        float2 sum2 = make_float2(0.f, 0.f);
-        uint32_t va[32], vb[32];
-        ptx::tmem_ld32(taddr, va);
-        tmem_ld_wait_for(va);
-        for (int c = 0; c < pieces; c += 2) {
-          if (c + 1 < pieces) ptx::tmem_ld32(taddr + (c + 1) * 32, vb);
-          add_key_piece(va, ctl.neg_lse + c * 32, ctl.limit + c * 32, masked, key, s.scale_log2, sum2);
-          if (c + 1 < pieces) {
-            tmem_ld_wait_for(vb);
-            if (c + 2 < pieces) ptx::tmem_ld32(taddr + (c + 2) * 32, va);
-            add_key_piece(vb, ctl.neg_lse + (c + 1) * 32, ctl.limit + (c + 1) * 32, masked, key, s.scale_log2, sum2);
-            if (c + 2 < pieces) tmem_ld_wait_for(va);
+      // Warpgroup w owns the K tiles of parity w (counted over the block's whole run): thread <-> key, all
+      // query-row columns.  Each warpgroup keeps its own copy of the per-column -lse and mask limits.
+      int tile_no = 0, q_gen = 0, loaded_gen = 0, min_limit = INT_MAX;
+      bool ok = true;
+      float* neg_lse = ctl.neg_lse[warp - 2];
+      int* limit = ctl.limit[warp - 2];
+      for (int u = 0; u < n_units && ok; ++u) {
+        const Unit un = ctl.units[u];
+        if (un.new_q) ++q_gen;
+        const int key_begin = un.kc * chunk_keys;
+        const int tiles = (min(un.n - key_begin, chunk_keys) + kTileKeys - 1) / kTileKeys;
+        const int first = (tile_no & 1) == wg ? 0 : 1;  // first tile of the unit that is this warpgroup's
+        if (first < tiles && loaded_gen != q_gen) {
+          // New query tile: this warp's copy of the per-column constants (no block-level barrier involved).
+          __syncwarp();
+          min_limit = INT_MAX;
+          for (int c = lane; c < kRowsPerCta; c += 32) {
+            const int f = un.rc * rows_per_chunk + c;
+            float nl = -INFINITY;
+            int lim = -1;
+            if (c < un.rows_here) {
+              const int r = f / s.group;
+              nl = -lse[(long long)(un.row0 + r) * s.hq + un.g * s.group + f % s.group];
+              lim = causal ? q_idx[un.row0 + r] : INT_MAX;
+              min_limit = min(min_limit, lim);
+            }
+            neg_lse[c] = nl;
+            limit[c] = lim;
           }
+          min_limit = __reduce_min_sync(0xFFFFFFFFu, min_limit);
+          __syncwarp();
+          loaded_gen = q_gen;
         }
-        ptx::tc_fence_before_sync();
-        ptx::mbar_arrive(ptx::smem_u32(&ctl.tmem_empty[buf]));
-        if (key < n) out[key] = sum2.x + sum2.y;
+        float* out = partial + (long long)(un.g * rc_max + un.rc) * s.total_tokens + un.tok0;
+        const int pieces = (un.rows_here + 31) / 32;
+        for (int t = first; t < tiles; t += 2) {
+          const int tn = tile_no + t, i = tn & 1;  // i == wg
+          ok = ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.tmem_full[i]), (tn >> 1) & 1, abort);
+          if (!ok) break;
+          ptx::tc_fence_after_sync();
+          const int key = key_begin + t * kTileKeys + my_lane;
+          const bool masked = causal && (key_begin + t * kTileKeys + kTileKeys - 1 > min_limit);
+          const uint32_t taddr = lane_addr + i * 256;
+          const float sum = masked ? sum_key_columns<true>(taddr, pieces, neg_lse, limit, key, s.scale_log2)
+                                   : sum_key_columns<false>(taddr, pieces, neg_lse, limit, key, s.scale_log2);
+          ptx::tc_fence_before_sync();
+          ptx::mbar_arrive(ptx::smem_u32(&ctl.tmem_empty[i]));
+          if (key < un.n) out[key] = sum;
+        }
+        tile_no += tiles;
       }
     }
   }
@@ -416,12 +598,12 @@ __global__ void __launch_bounds__(256) score_wide_merge_kernel(Shapes s, const i
 
 __global__ void __launch_bounds__(256) score_wide_finalize_kernel(Shapes s, const int32_t* __restrict__ cu_seqlens,
                                                                   const int32_t* __restrict__ cu_qlens, int rc_max,
-                                                                  const float* __restrict__ partial,
+                                                                  int rows_per_chunk, const float* __restrict__ partial,
                                                                   float* __restrict__ scores) {
   const int b = blockIdx.y;
   const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
   const int rows = cu_qlens[b + 1] - cu_qlens[b];
-  const int row_chunks = (rows * s.group + kRowsPerCta - 1) / kRowsPerCta;
+  const int row_chunks = (rows * s.group + rows_per_chunk - 1) / rows_per_chunk;
   const float inv = rows > 0 ? 1.0f / ((float)s.hq * (float)rows) : 0.f;
   for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < n; j += gridDim.x * blockDim.x) {
     float total = 0.f;
@@ -449,72 +631,87 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// K [N, Hkv, d] bf16 with element strides (k_st, k_sh, 1) as a rank-3 tensor (d, Hkv, N); one box is a
-// 64-element (128-byte) column block of 128 consecutive tokens of one KV head.
-bool make_k_map(const Shapes& s, const void* k, CUtensorMap* map) {
+// A [rows, heads, d] bf16 tensor with element strides (st, sh, 1) as a rank-3 tensor (d, heads, rows); a box
+// is a 64-element (128-byte) column block of `box_heads` heads of `box_rows` consecutive rows.
+bool make_map(const void* ptr, int dim, int heads, long long rows, long long st, long long sh, int box_heads, int box_rows,
+              CUtensorMap* map) {
   EncodeTiledFn encode = encode_tiled_fn();
-  if (!encode) return false;
-  const cuuint64_t dims[3] = {(cuuint64_t)s.dim, (cuuint64_t)s.hkv, (cuuint64_t)s.total_tokens};
-  const cuuint64_t strides[2] = {(cuuint64_t)s.k_sh * 2, (cuuint64_t)s.k_st * 2};
-  const cuuint32_t box[3] = {64, 1, (cuuint32_t)kTileKeys};
+  if (!encode || rows <= 0) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)dim, (cuuint64_t)heads, (cuuint64_t)rows};
+  const cuuint64_t strides[2] = {(cuuint64_t)sh * 2, (cuuint64_t)st * 2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)box_heads, (cuuint32_t)box_rows};
   const cuuint32_t elem[3] = {1, 1, 1};
-  return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(k), dims, strides, box, elem,
+  return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, elem,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 template <int DIM>
-cudaError_t run(const Shapes& s, const Workspace& w, const CUtensorMap& map, const uint16_t* q, const int32_t* q_idx,
+cudaError_t run(const Shapes& s, const Workspace& w, const CUtensorMap& k_map, const CUtensorMap& q_map, const int32_t* q_idx,
                 const int32_t* cu_qlens, const int32_t* cu_seqlens, float* scores_out, unsigned char* ws,
                 int32_t* device_status, cudaStream_t stream) {
   float2* stats = reinterpret_cast<float2*>(ws + w.stats_off);
   float* lse = reinterpret_cast<float*>(ws + w.lse_off);
   float* partial = reinterpret_cast<float*>(ws + w.partial_off);
+  const int rows_per_chunk = wide_rows_per_chunk(s.group);
   const int rc_max = wide_row_chunks(s.max_qlen, s.group);
-  // Key chunk per block: enough blocks for several waves of the 148 SMs, at most 16 tiles each.
-  const long long tiles_total = (long long)s.total_tokens / kTileKeys + s.batch;
-  long long chunk_tiles = tiles_total * s.hkv * rc_max / (kNumSMs * 6);
-  chunk_tiles = chunk_tiles < 1 ? 1 : (chunk_tiles > kMaxChunkTiles ? kMaxChunkTiles : chunk_tiles);
+  // One persistent block per SM.  Key chunks are sized so that a block gets about a dozen units (fine
+  // enough to balance, and never more than its table holds).
+  const long long tiles_upper = (long long)s.total_tokens / kTileKeys + s.batch;  // >= sum over sequences of ceil(n / 128)
+  const long long tile_units = tiles_upper * s.hkv * rc_max;
+  const int grid = (int)(tile_units < kNumSMs ? tile_units : kNumSMs);
+  long long chunk_tiles = (tile_units + (long long)grid * 14 - 1) / ((long long)grid * 14);
+  if (chunk_tiles < 1) chunk_tiles = 1;
+  // units <= hkv * rc_max * (tokens / chunk + batch); keep the per-block share within the table
+  while (((long long)s.hkv * rc_max * (s.total_tokens / (chunk_tiles * kTileKeys) + s.batch) + grid - 1) / grid + 1 > kMaxUnits)
+    ++chunk_tiles;
   const int chunk_keys = (int)chunk_tiles * kTileKeys;
   const int stat_chunks = (s.max_seqlen + chunk_keys - 1) / chunk_keys;
   const int smem = Layout<DIM>::kTotal;
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(score_wide_kernel<DIM, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(score_wide_kernel<DIM, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) return e;
-  const dim3 grid(stat_chunks, s.hkv * rc_max, s.batch);
-  score_wide_kernel<DIM, 1><<<grid, kThreads, smem, stream>>>(map, s, q, q_idx, cu_qlens, cu_seqlens, (int)chunk_tiles, stat_chunks,
-                                                              rc_max, stats, nullptr, nullptr, device_status);
+  score_wide_kernel<DIM, 1><<<grid, kThreads, smem, stream>>>(k_map, q_map, s, q_idx, cu_qlens, cu_seqlens, (int)chunk_tiles,
+                                                              stat_chunks, rc_max, rows_per_chunk, stats, nullptr, nullptr,
+                                                              device_status);
   const int warps = s.total_q * s.hq;
   score_wide_merge_kernel<<<(warps + 7) / 8, 256, 0, stream>>>(s, cu_qlens, cu_seqlens, stats, stat_chunks, chunk_keys, lse);
-  score_wide_kernel<DIM, 2><<<grid, kThreads, smem, stream>>>(map, s, q, q_idx, cu_qlens, cu_seqlens, (int)chunk_tiles, stat_chunks,
-                                                              rc_max, nullptr, lse, partial, device_status);
-  score_wide_finalize_kernel<<<dim3((s.max_seqlen + 255) / 256, s.batch), 256, 0, stream>>>(s, cu_seqlens, cu_qlens, rc_max, partial,
-                                                                                          scores_out);
+  score_wide_kernel<DIM, 2><<<grid, kThreads, smem, stream>>>(k_map, q_map, s, q_idx, cu_qlens, cu_seqlens, (int)chunk_tiles,
+                                                              stat_chunks, rc_max, rows_per_chunk, nullptr, lse, partial,
+                                                              device_status);
+  score_wide_finalize_kernel<<<dim3((s.max_seqlen + 255) / 256, s.batch), 256, 0, stream>>>(s, cu_seqlens, cu_qlens, rc_max,
+                                                                                          rows_per_chunk, partial, scores_out);
   count_launches(4);
   return cudaGetLastError();
 }
 
 }  // namespace
 
+// Query rows per block: whole TMA boxes of 8 scored rows x G heads, as many as fit in 256 rows.
+int wide_rows_per_chunk(int group) { return group >= 1 && group <= 32 ? kRowsPerCta / (8 * group) * (8 * group) : 0; }
+
 int wide_row_chunks(int max_qlen, int group) {
-  const int c = (max_qlen * group + kRowsPerCta - 1) / kRowsPerCta;
+  const int per = wide_rows_per_chunk(group);
+  if (per == 0) return 1;
+  const int c = (max_qlen * group + per - 1) / per;
   return c < 1 ? 1 : c;
 }
 
 bool score_wide_applies(const Shapes& s) {
-  return s.max_qlen >= 1 && s.total_q >= 1 && s.max_seqlen >= 1 && (s.dim == 64 || s.dim == 128) && s.k_st % 8 == 0 &&
-         s.k_sh % 8 == 0 && s.k_st > 0 && s.k_sh > 0 && (s.k_st >> 36) == 0 && (s.k_sh >> 36) == 0;
+  const auto ok_stride = [](long long v) { return v > 0 && v % 8 == 0 && (v >> 36) == 0; };
+  return s.max_qlen >= 1 && s.total_q >= 1 && s.max_seqlen >= 1 && (s.dim == 64 || s.dim == 128) && s.group <= 32 &&
+         ok_stride(s.k_st) && ok_stride(s.k_sh) && ok_stride(s.q_st) && ok_stride(s.q_sh);
 }
 
 cudaError_t launch_score_wide(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
                               const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
                               unsigned char* ws, int32_t* device_status, cudaStream_t stream, bool* used) {
-  CUtensorMap map;
-  *used = make_k_map(s, k, &map);
+  CUtensorMap k_map, q_map;
+  *used = make_map(k, s.dim, s.hkv, s.total_tokens, s.k_st, s.k_sh, 1, kTileKeys, &k_map) &&
+          make_map(q, s.dim, s.hq, s.total_q, s.q_st, s.q_sh, s.group, 8, &q_map);
   if (!*used) return cudaSuccess;  // the caller falls back to the CUDA-core path
-  const uint16_t* qq = static_cast<const uint16_t*>(q);
-  if (s.dim == 128) return run<128>(s, w, map, qq, q_idx, cu_qlens, cu_seqlens, scores_out, ws, device_status, stream);
-  return run<64>(s, w, map, qq, q_idx, cu_qlens, cu_seqlens, scores_out, ws, device_status, stream);
+  if (s.dim == 128) return run<128>(s, w, k_map, q_map, q_idx, cu_qlens, cu_seqlens, scores_out, ws, device_status, stream);
+  return run<64>(s, w, k_map, q_map, q_idx, cu_qlens, cu_seqlens, scores_out, ws, device_status, stream);
 }
 
 }  // namespace fastav
