@@ -137,7 +137,9 @@ Workspace plan_workspace(const fastav_params& p) {
   auto carve = [&](size_t bytes) { const size_t at = off; off = align_up(off + bytes, 256); return at; };
   const size_t rows_heads = (size_t)p.total_q * p.num_q_heads;
   w.stat_tiles = (p.max_seqlen + 63) / 64;
-  w.stats_off = carve(rows_heads * (size_t)w.stat_tiles * sizeof(float2));
+  // per (row, head): one (max, sum) per 64-key tile on the CUDA-core path, at most two per 128-key tile on the tensor-core path
+  const size_t stat_entries = (size_t)2 * ((p.max_seqlen + 127) / 128);
+  w.stats_off = carve(rows_heads * (stat_entries > (size_t)w.stat_tiles ? stat_entries : (size_t)w.stat_tiles) * sizeof(float2));
   w.lse_off = carve(rows_heads * sizeof(float));
   w.partial_off = carve((size_t)p.num_kv_heads * wide_row_chunks(p.max_qlen, p.num_q_heads / p.num_kv_heads) *
                         p.total_tokens * sizeof(float));

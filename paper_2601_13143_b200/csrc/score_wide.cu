@@ -9,14 +9,14 @@
 //   sweep 1 (S = Q K^T, TMEM lanes = query rows): each thread owns one row and keeps a running
 //            (max, sum 2^(z - max)) over the key chunk of its block -> stats, merged into a
 //            log2-sum-exp2 per (row, head);
-//   sweep 2 (S^T = K Q^T, TMEM lanes = keys): each thread owns one key and adds 2^(z - lse) over the
-//            block's query rows in a fixed column order -> partial[KV head, row chunk][token];
+//   sweep 2 (S^T = K Q^T, TMEM lanes = keys): each thread owns one key and adds 2^(z - lse) over 64 of
+//            the block's query rows in a fixed column order; four such sums -> partial[KV head, row chunk][token];
 //   finalize: scores = (sum of the partials in a fixed order) / (Hq R).
 //
 // One block = one (sequence, KV head, chunk of 256 query rows, chunk of key tiles).  Warp 0 streams
 // 128-key K tiles with TMA (128-byte swizzle) through a 4-stage mbarrier ring, warp 1 issues the MMAs
-// into a double-buffered accumulator, warps 2-9 (two warpgroups) read the accumulators back with
-// tcgen05.ld and do the softmax arithmetic.  The per-key arithmetic does not depend on the key's
+// into a double-buffered accumulator, warps 2-17 (four warpgroups) read the accumulators back with
+// tcgen05.ld and do the softmax arithmetic, part of the exponentials on the FMA pipe.  The per-key arithmetic does not depend on the key's
 // position, so equal keys get bit-equal scores; all sums have a fixed order, so runs are reproducible.
 // Every wait is bounded: a wait that expires makes the block give up, wait for its own copies, free its
 // tensor memory and set FASTAV_DEV_WAIT_EXPIRED.
@@ -27,9 +27,6 @@
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
-#ifndef FASTAV_EPI_SCALAR
-#define FASTAV_EPI_SCALAR 0
-#endif
 
 namespace fastav {
 namespace {
@@ -37,10 +34,11 @@ namespace {
 constexpr int kTileKeys = 128;    // keys per K tile
 constexpr int kRowsPerCta = 256;  // query rows (flat over scored row x head of the KV group) per block
 constexpr int kStages = 4;        // K tiles in flight
-constexpr int kThreads = 320;     // warp 0: TMA, warp 1: MMA, warps 2-9: softmax
+constexpr int kGroups = 4;        // softmax warpgroups: four warps per scheduler hide each other's latencies
+constexpr int kThreads = 64 + 128 * kGroups;  // warp 0: TMA, warp 1: MMA, warps 2-17: softmax
 constexpr int kTmemCols = 512;
 constexpr int kMaxUnits = 48;       // work units one block may be given (the host sizes key chunks accordingly)
-constexpr int kCtrlBytes = 20 * 1024;
+constexpr int kCtrlBytes = 16 * 1024;
 
 template <int DIM>
 struct Layout {
@@ -59,6 +57,36 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
   return d;
+}
+
+// 2^x for a pair of x <= ~0, computed on the FMA and integer pipes so that it can run next to the
+// exponentials the special-function unit is busy with: x = n + f with n the nearest integer (read off
+// the mantissa after adding 1.5 * 2^23), a cubic for 2^f on [-1/2, 1/2] (relative error below 7.5e-5),
+// and n added into the exponent field.  Inputs below -126 (including -inf) give about 2^-126.
+__device__ __forceinline__ float2 exp2_pair_fma(float2 x) {
+  const float kMagic = 12582912.f;
+  x.x = fmaxf(x.x, -126.f);
+  x.y = fmaxf(x.y, -126.f);
+  const float2 t = __fadd2_rn(x, make_float2(kMagic, kMagic));
+  const float2 n = __fadd2_rn(t, make_float2(-kMagic, -kMagic));
+  const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
+  float2 p = __ffma2_rn(f, make_float2(0.055171460f, 0.055171460f), make_float2(0.24261086f, 0.24261086f));
+  p = __ffma2_rn(p, f, make_float2(0.69326097f, 0.69326097f));
+  p = __ffma2_rn(p, f, make_float2(0.99992812f, 0.99992812f));
+  return make_float2(__int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23)),
+                     __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23)));
+}
+
+// The softmax is bound by exponentials, so they are split over two pipes: of the 8 column pairs of every
+// 16-column block, the pairs in kFmaPairs go through exp2_pair_fma, the others through the special-function unit.
+#ifndef FASTAV_FMA_PAIRS
+#define FASTAV_FMA_PAIRS 0x92  // pairs 1, 4, 7: three of eight
+#endif
+constexpr unsigned kFmaPairs = FASTAV_FMA_PAIRS;
+
+__device__ __forceinline__ float2 exp2_pair(float2 x, int pair) {
+  if ((kFmaPairs >> (pair & 7)) & 1u) return exp2_pair_fma(x);
+  return make_float2(ptx::ex2_approx(x.x), ptx::ex2_approx(x.y));
 }
 
 // tcgen05.wait::ld, tied to the registers of the load it completes so that no use can move above it.
@@ -93,20 +121,10 @@ __device__ __forceinline__ void fold_row_piece(const uint32_t (&v)[32], int boun
   sum2.y *= corr;
   zmax = newmax;
   const float shift = -ref * scale;
-#if FASTAV_EPI_SCALAR
-#pragma unroll
-  for (int j = 0; j < 32; j += 2) {
-    sum2.x += ptx::ex2_approx(fmaf(z[j], scale, shift));
-    sum2.y += ptx::ex2_approx(fmaf(z[j + 1], scale, shift));
-  }
-#else
   const float2 sc = make_float2(scale, scale), sh = make_float2(shift, shift);
 #pragma unroll
-  for (int j = 0; j < 32; j += 2) {
-    const float2 x = __ffma2_rn(make_float2(z[j], z[j + 1]), sc, sh);
-    sum2 = __fadd2_rn(sum2, make_float2(ptx::ex2_approx(x.x), ptx::ex2_approx(x.y)));
-  }
-#endif
+  for (int j = 0; j < 32; j += 2)
+    sum2 = __fadd2_rn(sum2, exp2_pair(__ffma2_rn(make_float2(z[j], z[j + 1]), sc, sh), j / 2));
 }
 
 __device__ __forceinline__ void fold_row_piece_any(const uint32_t (&v)[32], int bound, float scale, float& zmax, float2& sum2) {
@@ -120,57 +138,37 @@ __device__ __forceinline__ void fold_row_piece_any(const uint32_t (&v)[32], int 
 template <bool MASKED>
 __device__ __forceinline__ void add_key_piece(const uint32_t (&v)[32], const float* neg_lse, const int* limit, int key,
                                               float scale, float2& sum2) {
+  const float2 sc = make_float2(scale, scale);
 #pragma unroll
   for (int j = 0; j < 32; j += 4) {
     const float4 nl = *reinterpret_cast<const float4*>(neg_lse + j);
-#if FASTAV_EPI_SCALAR
-    float p0 = ptx::ex2_approx(fmaf(__uint_as_float(v[j]), scale, nl.x));
-    float p1 = ptx::ex2_approx(fmaf(__uint_as_float(v[j + 1]), scale, nl.y));
-    float p2 = ptx::ex2_approx(fmaf(__uint_as_float(v[j + 2]), scale, nl.z));
-    float p3 = ptx::ex2_approx(fmaf(__uint_as_float(v[j + 3]), scale, nl.w));
-#else
-    const float2 sc = make_float2(scale, scale);
-    const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(v[j]), __uint_as_float(v[j + 1])), sc, make_float2(nl.x, nl.y));
-    const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])), sc, make_float2(nl.z, nl.w));
-    float p0 = ptx::ex2_approx(x0.x), p1 = ptx::ex2_approx(x0.y), p2 = ptx::ex2_approx(x1.x), p3 = ptx::ex2_approx(x1.y);
-#endif
+    float2 p0 = exp2_pair(__ffma2_rn(make_float2(__uint_as_float(v[j]), __uint_as_float(v[j + 1])), sc, make_float2(nl.x, nl.y)), j / 2);
+    float2 p1 = exp2_pair(__ffma2_rn(make_float2(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])), sc, make_float2(nl.z, nl.w)), j / 2 + 1);
     if (MASKED) {
       const int4 lim = *reinterpret_cast<const int4*>(limit + j);
-      p0 = key <= lim.x ? p0 : 0.f;
-      p1 = key <= lim.y ? p1 : 0.f;
-      p2 = key <= lim.z ? p2 : 0.f;
-      p3 = key <= lim.w ? p3 : 0.f;
+      p0.x = key <= lim.x ? p0.x : 0.f;
+      p0.y = key <= lim.y ? p0.y : 0.f;
+      p1.x = key <= lim.z ? p1.x : 0.f;
+      p1.y = key <= lim.w ? p1.y : 0.f;
     }
-#if FASTAV_EPI_SCALAR
-    sum2.x += p0; sum2.y += p1; sum2.x += p2; sum2.y += p3;
-#else
-    sum2 = __fadd2_rn(sum2, make_float2(p0, p1));
-    sum2 = __fadd2_rn(sum2, make_float2(p2, p3));
-#endif
+    sum2 = __fadd2_rn(sum2, p0);
+    sum2 = __fadd2_rn(sum2, p1);
   }
 }
 
-// Sweep 2, all query-row columns of one key: the accumulator is read 32 columns at a time, the next
-// read in flight while the current one is summed.
+// Sweep 2, the (at most 64) query-row columns of one key that belong to this warpgroup.
 template <bool MASKED>
 __device__ __forceinline__ float sum_key_columns(uint32_t taddr, int pieces, const float* neg_lse, const int* limit, int key,
                                                  float scale) {
   float2 sum2 = make_float2(0.f, 0.f);
-  uint32_t va[32], vb[32];
-  ptx::tmem_ld32(taddr, va);
-  int c = 0;
-#pragma unroll 1
-  for (; c + 2 <= pieces; c += 2) {
-    tmem_ld_wait_for(va);
-    ptx::tmem_ld32(taddr + (c + 1) * 32, vb);
-    add_key_piece<MASKED>(va, neg_lse + c * 32, limit + c * 32, key, scale, sum2);
-    tmem_ld_wait_for(vb);
-    if (c + 2 < pieces) ptx::tmem_ld32(taddr + (c + 2) * 32, va);
-    add_key_piece<MASKED>(vb, neg_lse + (c + 1) * 32, limit + (c + 1) * 32, key, scale, sum2);
-  }
-  if (c < pieces) {
-    tmem_ld_wait_for(va);
-    add_key_piece<MASKED>(va, neg_lse + c * 32, limit + c * 32, key, scale, sum2);
+  uint32_t v[32];
+  ptx::tmem_ld32(taddr, v);
+  tmem_ld_wait_for(v);
+  add_key_piece<MASKED>(v, neg_lse, limit, key, scale, sum2);
+  if (pieces > 1) {  // the other warps of the scheduler cover this load's latency
+    ptx::tmem_ld32(taddr + 32, v);
+    tmem_ld_wait_for(v);
+    add_key_piece<MASKED>(v, neg_lse + 32, limit + 32, key, scale, sum2);
   }
   return sum2.x + sum2.y;
 }
@@ -188,13 +186,15 @@ struct Control {
   uint64_t full_k[kStages], empty_k[kStages];
   uint64_t q_ready, q_free;
   uint64_t tmem_full[4], tmem_empty[4];
+  uint64_t sums_ready[2];  // sweep 2: warpgroups 1-3 have published their partial sums of accumulator i
   uint32_t tmem_base;
   int abort;
   int n_units;
   int start_b, start_off;
   int warp_sums[kThreads / 32];
-  alignas(16) float neg_lse[8][kRowsPerCta];  // sweep 2, per softmax warp: -lse of each query-row column (-inf: padding)
-  alignas(16) int limit[8][kRowsPerCta];      // sweep 2, per softmax warp: last key each column's row may see
+  alignas(16) float neg_lse[4 * kGroups][64];  // sweep 2, per softmax warp: -lse of its query-row columns (-inf: padding)
+  alignas(16) int limit[4 * kGroups][64];      // sweep 2, per softmax warp: last key each column's row may see
+  float sums[2][kGroups - 1][kTileKeys];       // sweep 2: per accumulator, the partial sums of warpgroups 1-3
   Unit units[kMaxUnits];
 };
 static_assert(sizeof(Control) <= kCtrlBytes, "control block must fit its slot");
@@ -284,15 +284,18 @@ score_wide_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
   if (threadIdx.x == 0) {
     // Walk the units of this block and write them down for every role.
     int b = ctl.start_b, off = ctl.start_off, count = 0, prev_b = -1, prev_grc = -1;
+    int tok0 = 0, n = 0, row0 = 0, flat_rows = 0, row_chunks = 0, key_chunks = 0, loaded_b = -1;
     for (int u = u0; u < u1 && count < kMaxUnits; ++u) {
-      int tok0, n, row0, flat_rows, row_chunks, key_chunks;
       for (;;) {
-        tok0 = cu_seqlens[b];
-        n = cu_seqlens[b + 1] - tok0;
-        row0 = cu_qlens[b];
-        flat_rows = (cu_qlens[b + 1] - row0) * s.group;
-        row_chunks = (flat_rows + rows_per_chunk - 1) / rows_per_chunk;
-        key_chunks = (n + chunk_keys - 1) / chunk_keys;
+        if (b != loaded_b) {  // the (slow, dependent) global loads happen once per sequence
+          tok0 = cu_seqlens[b];
+          n = cu_seqlens[b + 1] - tok0;
+          row0 = cu_qlens[b];
+          flat_rows = (cu_qlens[b + 1] - row0) * s.group;
+          row_chunks = (flat_rows + rows_per_chunk - 1) / rows_per_chunk;
+          key_chunks = (n + chunk_keys - 1) / chunk_keys;
+          loaded_b = b;
+        }
         if (n > 0 && flat_rows > 0 && off < s.hkv * row_chunks * key_chunks) break;
         ++b;  // sequence exhausted (or empty): on to the next one
         off = 0;
@@ -316,8 +319,10 @@ score_wide_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
     ptx::mbar_init(ptx::smem_u32(&ctl.q_free), 1);
     for (int i = 0; i < 4; ++i) {
       ptx::mbar_init(ptx::smem_u32(&ctl.tmem_full[i]), 1);
-      ptx::mbar_init(ptx::smem_u32(&ctl.tmem_empty[i]), 128);
+      // sweep 1: accumulator (e, i) is read by the two warpgroups of row tile e; sweep 2: accumulator i by all four
+      ptx::mbar_init(ptx::smem_u32(&ctl.tmem_empty[i]), SWEEP == 1 ? 256 : 128 * kGroups);
     }
+    for (int i = 0; i < 2; ++i) ptx::mbar_init(ptx::smem_u32(&ctl.sums_ready[i]), 128 * (kGroups - 1));
     ctl.abort = 0;
     ptx::fence_barrier_init();
     ptx::prefetch_tensormap(&k_map);
@@ -450,15 +455,16 @@ score_wide_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
       }
     }
   } else {
-    // ---- softmax warps ---------------------------------------------------------------------------
-    const int wg = (warp - 2) >> 2;           // warpgroup 0 / 1
+    // ---- softmax warps: four warpgroups, so that every scheduler has four of them to pick from ---------
+    const int wg = (warp - 2) >> 2;           // warpgroup 0..3
     const int quarter = warp & 3;             // the 32 TMEM lanes this warp may read
     const int my_lane = quarter * 32 + lane;  // row (sweep 1) or key (sweep 2) inside the tile
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
 
     if constexpr (SWEEP == 1) {
-      // Warpgroup e owns the rows of 128-row tile e: thread <-> row.
-      const int e = wg;
+      // Warpgroup (e, h) owns the rows of 128-row tile e and the keys [64 h, 64 h + 64) of every K tile:
+      // thread <-> row, its running (max, sum) over that half of the keys -> one stats entry per half.
+      const int e = wg & 1, h = wg >> 1;
       int uses = 0;
       bool ok = true;
       for (int u = 0; u < n_units && ok; ++u) {
@@ -477,51 +483,46 @@ score_wide_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
           ok = ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.tmem_full[i * 2 + e]), (uses >> 1) & 1, abort);
           if (!ok) break;
           ptx::tc_fence_after_sync();
-          const int bound = last_visible - (key_begin + t * kTileKeys);  // columns 0..bound of this tile are visible
-          const uint32_t taddr = lane_addr + i * 256 + e * 128;
+          const int bound = last_visible - (key_begin + t * kTileKeys + h * 64);  // columns 0..bound of this half are visible
+          const uint32_t taddr = lane_addr + i * 256 + e * 128 + h * 64;
           uint32_t va[32], vb[32];
           ptx::tmem_ld32(taddr, va);
           tmem_ld_wait_for(va);
           ptx::tmem_ld32(taddr + 32, vb);
           fold_row_piece_any(va, bound, s.scale_log2, zmax, sum2);
           tmem_ld_wait_for(vb);
-          ptx::tmem_ld32(taddr + 64, va);
-          fold_row_piece_any(vb, bound - 32, s.scale_log2, zmax, sum2);
-          tmem_ld_wait_for(va);
-          ptx::tmem_ld32(taddr + 96, vb);
-          fold_row_piece_any(va, bound - 64, s.scale_log2, zmax, sum2);
-          tmem_ld_wait_for(vb);
           ptx::tc_fence_before_sync();
           ptx::mbar_arrive(ptx::smem_u32(&ctl.tmem_empty[i * 2 + e]));  // the accumulator may be overwritten
-          fold_row_piece_any(vb, bound - 96, s.scale_log2, zmax, sum2);
+          fold_row_piece_any(vb, bound - 32, s.scale_log2, zmax, sum2);
         }
         if (ok && row_valid) {
           const long long rh = (long long)(un.row0 + r) * s.hq + un.g * s.group + f % s.group;
-          stats[rh * stat_chunks + un.kc] = make_float2(zmax * s.scale_log2, sum2.x + sum2.y);
+          stats[rh * stat_chunks + un.kc * 2 + h] = make_float2(zmax * s.scale_log2, sum2.x + sum2.y);
         }
       }
     } else {
-      // Warpgroup w owns the K tiles of parity w (counted over the block's whole run): thread <-> key, all
-      // query-row columns.  Each warpgroup keeps its own copy of the per-column -lse and mask limits.
-      int tile_no = 0, q_gen = 0, loaded_gen = 0, min_limit = INT_MAX;
+      // Every K tile is shared by the four warpgroups: thread <-> key, warpgroup w sums the query-row columns
+      // [64 w, 64 w + 64); warpgroups 1-3 publish their sums in shared memory and warpgroup 0 adds them in a
+      // fixed order and writes the partial.  Each warp keeps its own copy of the per-column -lse and mask
+      // limits (no block-level barrier between softmax warps).
+      int tile_no = 0, min_limit = INT_MAX;
       bool ok = true;
       float* neg_lse = ctl.neg_lse[warp - 2];
       int* limit = ctl.limit[warp - 2];
       for (int u = 0; u < n_units && ok; ++u) {
         const Unit un = ctl.units[u];
-        if (un.new_q) ++q_gen;
         const int key_begin = un.kc * chunk_keys;
         const int tiles = (min(un.n - key_begin, chunk_keys) + kTileKeys - 1) / kTileKeys;
-        const int first = (tile_no & 1) == wg ? 0 : 1;  // first tile of the unit that is this warpgroup's
-        if (first < tiles && loaded_gen != q_gen) {
-          // New query tile: this warp's copy of the per-column constants (no block-level barrier involved).
+        const int my_cols = max(0, min(64, un.rows_here - wg * 64));  // columns of this warpgroup that exist
+        const int pieces = (my_cols + 31) / 32;
+        if (un.new_q) {
           __syncwarp();
           min_limit = INT_MAX;
-          for (int c = lane; c < kRowsPerCta; c += 32) {
-            const int f = un.rc * rows_per_chunk + c;
+          for (int c = lane; c < 64; c += 32) {
+            const int f = un.rc * rows_per_chunk + wg * 64 + c;
             float nl = -INFINITY;
             int lim = -1;
-            if (c < un.rows_here) {
+            if (c < my_cols) {
               const int r = f / s.group;
               nl = -lse[(long long)(un.row0 + r) * s.hq + un.g * s.group + f % s.group];
               lim = causal ? q_idx[un.row0 + r] : INT_MAX;
@@ -532,25 +533,35 @@ score_wide_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
           }
           min_limit = __reduce_min_sync(0xFFFFFFFFu, min_limit);
           __syncwarp();
-          loaded_gen = q_gen;
         }
         float* out = partial + (long long)(un.g * rc_max + un.rc) * s.total_tokens + un.tok0;
-        const int pieces = (un.rows_here + 31) / 32;
-        for (int t = first; t < tiles; t += 2) {
-          const int tn = tile_no + t, i = tn & 1;  // i == wg
-          ok = ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.tmem_full[i]), (tn >> 1) & 1, abort);
+        for (int t = 0; t < tiles; ++t, ++tile_no) {
+          const int i = tile_no & 1;
+          const uint32_t parity = (tile_no >> 1) & 1;
+          ok = ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.tmem_full[i]), parity, abort);
           if (!ok) break;
           ptx::tc_fence_after_sync();
           const int key = key_begin + t * kTileKeys + my_lane;
           const bool masked = causal && (key_begin + t * kTileKeys + kTileKeys - 1 > min_limit);
-          const uint32_t taddr = lane_addr + i * 256;
-          const float sum = masked ? sum_key_columns<true>(taddr, pieces, neg_lse, limit, key, s.scale_log2)
-                                   : sum_key_columns<false>(taddr, pieces, neg_lse, limit, key, s.scale_log2);
+          const uint32_t taddr = lane_addr + i * 256 + wg * 64;
+          float sum = 0.f;
+          if (pieces > 0)
+            sum = masked ? sum_key_columns<true>(taddr, pieces, neg_lse, limit, key, s.scale_log2)
+                         : sum_key_columns<false>(taddr, pieces, neg_lse, limit, key, s.scale_log2);
+          if (wg > 0) {
+            // sums[i] is free again: warpgroup 0 read it before it released accumulator i two tiles ago
+            ctl.sums[i][wg - 1][my_lane] = sum;
+            ptx::mbar_arrive(ptx::smem_u32(&ctl.sums_ready[i]));
+          } else {
+            ok = ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.sums_ready[i]), parity, abort);
+            if (!ok) break;
+#pragma unroll
+            for (int w = 0; w < kGroups - 1; ++w) sum += ctl.sums[i][w][my_lane];
+            if (key < un.n) out[key] = sum;
+          }
           ptx::tc_fence_before_sync();
           ptx::mbar_arrive(ptx::smem_u32(&ctl.tmem_empty[i]));
-          if (key < un.n) out[key] = sum;
         }
-        tile_no += tiles;
       }
     }
   }
@@ -579,7 +590,7 @@ __global__ void __launch_bounds__(256) score_wide_merge_kernel(Shapes s, const i
     if (cu_qlens[mid] <= row) lo = mid; else hi = mid;
   }
   const int n = cu_seqlens[lo + 1] - cu_seqlens[lo];
-  const int chunks = (n + chunk_keys - 1) / chunk_keys;
+  const int chunks = 2 * ((n + chunk_keys - 1) / chunk_keys);  // one entry per 64-key half of every tile run
   const float2* mine = stats + (long long)w * stat_chunks;
   float m = -INFINITY;
   for (int t = lane; t < chunks; t += 32) m = fmaxf(m, mine[t].x);
@@ -666,7 +677,7 @@ cudaError_t run(const Shapes& s, const Workspace& w, const CUtensorMap& k_map, c
   while (((long long)s.hkv * rc_max * (s.total_tokens / (chunk_tiles * kTileKeys) + s.batch) + grid - 1) / grid + 1 > kMaxUnits)
     ++chunk_tiles;
   const int chunk_keys = (int)chunk_tiles * kTileKeys;
-  const int stat_chunks = (s.max_seqlen + chunk_keys - 1) / chunk_keys;
+  const int stat_chunks = 2 * ((s.max_seqlen + chunk_keys - 1) / chunk_keys);  // (max, sum) entries per (row, head)
   const int smem = Layout<DIM>::kTotal;
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(score_wide_kernel<DIM, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) return e;
