@@ -76,4 +76,32 @@ void count_launches(int n);
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// ---- programmatic dependent launch ----------------------------------------------------------------
+// The kernels of one prune call form a chain in which each reads what its predecessor wrote.  They
+// are launched with programmatic stream serialization: a kernel lets its successor start early
+// (pdl_trigger, first thing) so that the successor's set-up overlaps this kernel's tail, and every
+// block of the successor calls pdl_wait -- which returns once the predecessor has completed and its
+// writes are visible -- before it touches global memory another kernel may have written, or writes
+// global memory another kernel may still read.  Every block waits before it exits, so completion of a
+// kernel implies completion of all its predecessors.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 }  // namespace fastav

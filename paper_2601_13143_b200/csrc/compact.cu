@@ -40,6 +40,8 @@ __global__ void __launch_bounds__(kThreads) compact_rows_kernel(Shapes s, RowStr
                                                                 const int32_t* __restrict__ cu_keep,
                                                                 const int32_t* __restrict__ cu_seqlens,
                                                                 int32_t* device_status) {
+  pdl_trigger();
+  pdl_wait();  // keep_idx and cu_keep are the previous kernel's output
   // 16-byte chunks per output row: [hidden | K heads | V heads]
   const int per_head = s.dim >> 3;
   const int n_hidden = t.hidden_in ? (s.hidden >> 3) : 0;
@@ -111,9 +113,10 @@ cudaError_t launch_compact(const Shapes& s, const int32_t* keep_idx, const int32
                pos_in,                                  pos_out};
   int blocks = kNumSMs * 8;
   if (blocks > s.total_keep) blocks = s.total_keep;
-  compact_rows_kernel<<<blocks, kThreads, 0, stream>>>(s, t, keep_idx, cu_keep, cu_seqlens, device_status);
+  const cudaError_t e = launch_chained(compact_rows_kernel, dim3(blocks), dim3(kThreads), 0, stream, s, t, keep_idx, cu_keep,
+                                       cu_seqlens, device_status);
   count_launches(1);
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace fastav

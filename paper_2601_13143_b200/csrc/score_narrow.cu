@@ -40,6 +40,8 @@ score_narrow_logits_kernel(Shapes s, const uint16_t* __restrict__ q, const int32
   constexpr int kHalvings = ROWS == 8 ? 3 : 2;  // butterfly steps that halve the row set
   constexpr int kPlainBits = (kLanes == 16 ? 4 : 3) - kHalvings;
 
+  pdl_trigger();
+  pdl_wait();  // q and k may be what the previous kernel wrote; the logits may still be read by it
   const int b = blockIdx.z;
   const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
   const int key_begin = blockIdx.x * chunk_keys;
@@ -131,6 +133,8 @@ __global__ void __launch_bounds__(256) score_narrow_stats_kernel(Shapes s, const
                                                                  const float* __restrict__ logits, int rq,
                                                                  float* __restrict__ lse) {
   __shared__ float red[8];
+  pdl_trigger();
+  pdl_wait();
   const int b = blockIdx.y, head = blockIdx.x / rq, r = blockIdx.x % rq;
   const int row0 = cu_qlens[b], rows = min(cu_qlens[b + 1] - row0, rq);
   if (r >= rows) return;
@@ -168,6 +172,8 @@ __global__ void __launch_bounds__(256) score_narrow_finalize_kernel(Shapes s, co
                                                                     const float* __restrict__ lse,
                                                                     float* __restrict__ scores) {
   extern __shared__ float lse_sh[];  // [Hq][rows]
+  pdl_trigger();
+  pdl_wait();
   const int b = blockIdx.y;
   const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
   if ((int)(blockIdx.x * blockDim.x) >= n) return;
@@ -189,7 +195,7 @@ __global__ void __launch_bounds__(256) score_narrow_finalize_kernel(Shapes s, co
 }
 
 template <int DIM, int ROWS>
-void launch_logits(const Shapes& s, const uint16_t* q, const int32_t* q_idx, const int32_t* cu_qlens, const uint16_t* k,
+cudaError_t launch_logits(const Shapes& s, const uint16_t* q, const int32_t* q_idx, const int32_t* cu_qlens, const uint16_t* k,
                    const int32_t* cu_seqlens, float* logits, int rq, cudaStream_t stream) {
   constexpr int kGroups = kThreads / (DIM / 8);
   // One block covers `hb` KV heads so that a step of the block reads whole contiguous token rows.
@@ -204,8 +210,8 @@ void launch_logits(const Shapes& s, const uint16_t* q, const int32_t* q_idx, con
   if (chunk < quantum) chunk = quantum;
   if (chunk > 8 * quantum) chunk = 8 * quantum;
   const dim3 grid((unsigned)((s.max_seqlen + chunk - 1) / chunk), s.hkv / hb, s.batch);
-  score_narrow_logits_kernel<DIM, ROWS><<<grid, kThreads, 0, stream>>>(s, q, q_idx, cu_qlens, k, cu_seqlens, logits, rq, hb,
-                                                                      (int)chunk);
+  return launch_chained(score_narrow_logits_kernel<DIM, ROWS>, grid, dim3(kThreads), 0, stream, s, q, q_idx, cu_qlens, k, cu_seqlens,
+                        logits, rq, hb, (int)chunk);
 }
 
 }  // namespace
@@ -221,16 +227,22 @@ cudaError_t launch_score_narrow(const Shapes& s, const Workspace& w, const void*
   float* lse = reinterpret_cast<float*>(ws + w.lse_off);
   const int rq = s.max_qlen;
   const bool four = s.max_qlen * s.group <= 4;
+  cudaError_t e;
   if (s.dim == 128) {
-    if (four) launch_logits<128, 4>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, stream);
-    else launch_logits<128, 8>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, stream);
+    e = four ? launch_logits<128, 4>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, stream)
+             : launch_logits<128, 8>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, stream);
   } else {
-    if (four) launch_logits<64, 4>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, stream);
-    else launch_logits<64, 8>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, stream);
+    e = four ? launch_logits<64, 4>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, stream)
+             : launch_logits<64, 8>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, stream);
   }
-  score_narrow_stats_kernel<<<dim3(s.hq * rq, s.batch), 256, 0, stream>>>(s, cu_qlens, cu_seqlens, logits, rq, lse);
-  score_narrow_finalize_kernel<<<dim3((s.max_seqlen + 255) / 256, s.batch), 256, s.hq * rq * sizeof(float), stream>>>(
-      s, cu_qlens, cu_seqlens, logits, rq, lse, scores_out);
+  if (e != cudaSuccess) return e;
+  if ((e = launch_chained(score_narrow_stats_kernel, dim3(s.hq * rq, s.batch), dim3(256), 0, stream, s, cu_qlens, cu_seqlens,
+                          (const float*)logits, rq, lse)) != cudaSuccess)
+    return e;
+  if ((e = launch_chained(score_narrow_finalize_kernel, dim3((s.max_seqlen + 255) / 256, s.batch), dim3(256),
+                          s.hq * rq * sizeof(float), stream, s, cu_qlens, cu_seqlens, (const float*)logits, rq, (const float*)lse,
+                          scores_out)) != cudaSuccess)
+    return e;
   count_launches(3);
   return cudaGetLastError();
 }

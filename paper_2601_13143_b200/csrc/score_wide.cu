@@ -231,6 +231,7 @@ score_wide_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
                   int32_t* device_status) {
   using L = Layout<DIM>;
   extern __shared__ unsigned char smem_raw[];
+  pdl_trigger();
   const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_raw + (base - ptx::smem_u32(smem_raw));
   Control& ctl = *reinterpret_cast<Control*>(base_ptr + L::kCtrlOff);
@@ -251,7 +252,10 @@ score_wide_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
   }
   const int u0 = (int)((long long)total_units * blockIdx.x / gridDim.x);
   const int u1 = (int)((long long)total_units * (blockIdx.x + 1) / gridDim.x);
-  if (u1 <= u0) return;  // uniform: nothing for this block
+  if (u1 <= u0) {  // uniform: nothing for this block
+    pdl_wait();
+    return;
+  }
   {
     int before = 0;  // units of the sequences before the current batch slice
     for (int b0 = 0; b0 < s.batch; b0 += kThreads) {
@@ -345,6 +349,7 @@ score_wide_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
   if (warp == 0) {
     // ---- TMA producer: one elected lane streams query tiles and K tiles ---------------------------
     if (lane == 0) {
+      if constexpr (SWEEP == 1) pdl_wait();  // q and k may be what the previous kernel in the stream wrote
       int tile_no = 0, q_gen = 0;  // K tiles / query tiles issued so far
       bool ok = true;
       for (int u = 0; u < n_units && ok; ++u) {
@@ -460,6 +465,7 @@ score_wide_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
     const int quarter = warp & 3;             // the 32 TMEM lanes this warp may read
     const int my_lane = quarter * 32 + lane;  // row (sweep 1) or key (sweep 2) inside the tile
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
+    pdl_wait();  // before the first read of lse (sweep 2) and the first write of stats / partial
 
     if constexpr (SWEEP == 1) {
       // Warpgroup (e, h) owns the rows of 128-row tile e and the keys [64 h, 64 h + 64) of every K tile:
@@ -581,6 +587,8 @@ __global__ void __launch_bounds__(256) score_wide_merge_kernel(Shapes s, const i
                                                                const int32_t* __restrict__ cu_seqlens,
                                                                const float2* __restrict__ stats, int stat_chunks,
                                                                int chunk_keys, float* __restrict__ lse) {
+  pdl_trigger();
+  pdl_wait();
   const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (w >= s.total_q * s.hq) return;
   const int row = w / s.hq;
@@ -611,10 +619,12 @@ __global__ void __launch_bounds__(256) score_wide_finalize_kernel(Shapes s, cons
                                                                   const int32_t* __restrict__ cu_qlens, int rc_max,
                                                                   int rows_per_chunk, const float* __restrict__ partial,
                                                                   float* __restrict__ scores) {
+  pdl_trigger();
   const int b = blockIdx.y;
   const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
   const int rows = cu_qlens[b + 1] - cu_qlens[b];
   const int row_chunks = (rows * s.group + rows_per_chunk - 1) / rows_per_chunk;
+  pdl_wait();
   const float inv = rows > 0 ? 1.0f / ((float)s.hq * (float)rows) : 0.f;
   for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < n; j += gridDim.x * blockDim.x) {
     float total = 0.f;
@@ -682,16 +692,21 @@ cudaError_t run(const Shapes& s, const Workspace& w, const CUtensorMap& k_map, c
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(score_wide_kernel<DIM, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(score_wide_kernel<DIM, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) return e;
-  score_wide_kernel<DIM, 1><<<grid, kThreads, smem, stream>>>(k_map, q_map, s, q_idx, cu_qlens, cu_seqlens, (int)chunk_tiles,
-                                                              stat_chunks, rc_max, rows_per_chunk, stats, nullptr, nullptr,
-                                                              device_status);
+  if ((e = launch_chained(score_wide_kernel<DIM, 1>, dim3(grid), dim3(kThreads), smem, stream, k_map, q_map, s, q_idx, cu_qlens,
+                          cu_seqlens, (int)chunk_tiles, stat_chunks, rc_max, rows_per_chunk, stats, (const float*)nullptr,
+                          (float*)nullptr, device_status)) != cudaSuccess)
+    return e;
   const int warps = s.total_q * s.hq;
-  score_wide_merge_kernel<<<(warps + 7) / 8, 256, 0, stream>>>(s, cu_qlens, cu_seqlens, stats, stat_chunks, chunk_keys, lse);
-  score_wide_kernel<DIM, 2><<<grid, kThreads, smem, stream>>>(k_map, q_map, s, q_idx, cu_qlens, cu_seqlens, (int)chunk_tiles,
-                                                              stat_chunks, rc_max, rows_per_chunk, nullptr, lse, partial,
-                                                              device_status);
-  score_wide_finalize_kernel<<<dim3((s.max_seqlen + 255) / 256, s.batch), 256, 0, stream>>>(s, cu_seqlens, cu_qlens, rc_max,
-                                                                                          rows_per_chunk, partial, scores_out);
+  if ((e = launch_chained(score_wide_merge_kernel, dim3((warps + 7) / 8), dim3(256), 0, stream, s, cu_qlens, cu_seqlens,
+                          (const float2*)stats, stat_chunks, chunk_keys, lse)) != cudaSuccess)
+    return e;
+  if ((e = launch_chained(score_wide_kernel<DIM, 2>, dim3(grid), dim3(kThreads), smem, stream, k_map, q_map, s, q_idx, cu_qlens,
+                          cu_seqlens, (int)chunk_tiles, stat_chunks, rc_max, rows_per_chunk, (float2*)nullptr, (const float*)lse,
+                          partial, device_status)) != cudaSuccess)
+    return e;
+  if ((e = launch_chained(score_wide_finalize_kernel, dim3((s.max_seqlen + 255) / 256, s.batch), dim3(256), 0, stream, s,
+                          cu_seqlens, cu_qlens, rc_max, rows_per_chunk, (const float*)partial, scores_out)) != cudaSuccess)
+    return e;
   count_launches(4);
   return cudaGetLastError();
 }

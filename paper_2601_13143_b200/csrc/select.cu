@@ -47,6 +47,8 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
   SelectShared& sh = *reinterpret_cast<SelectShared*>(smem_raw);
   unsigned* keys = kKeysInShared ? reinterpret_cast<unsigned*>(smem_raw + sizeof(SelectShared)) : nullptr;
 
+  pdl_trigger();
+  pdl_wait();  // the scores are the previous kernel's output
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
   if (!kKeysInShared) keys = keys_global + tok0;
@@ -183,18 +185,18 @@ cudaError_t launch_select(const Shapes& s, const Workspace& w, const float* scor
   const size_t fixed = sizeof(SelectShared);
   const size_t want = fixed + (size_t)s.max_seqlen * sizeof(unsigned);
   constexpr size_t kMaxDynamic = 227 * 1024 - 1024;
+  cudaError_t e;
   if (want <= kMaxDynamic) {
-    cudaError_t e = cudaFuncSetAttribute(select_topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynamic);
+    e = cudaFuncSetAttribute(select_topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynamic);
     if (e != cudaSuccess) return e;
-    select_topk_kernel<true><<<s.batch, kThreads, want, stream>>>(s, scores, cu_seqlens, keep_counts, protect, q_idx,
-                                                                  cu_qlens, keep_idx, cu_keep, nullptr, device_status);
+    e = launch_chained(select_topk_kernel<true>, dim3(s.batch), dim3(kThreads), want, stream, s, scores, cu_seqlens, keep_counts,
+                       protect, q_idx, cu_qlens, keep_idx, cu_keep, (unsigned*)nullptr, device_status);
   } else {
-    select_topk_kernel<false><<<s.batch, kThreads, fixed, stream>>>(s, scores, cu_seqlens, keep_counts, protect, q_idx,
-                                                                    cu_qlens, keep_idx, cu_keep,
-                                                                    reinterpret_cast<unsigned*>(ws + w.keys_off), device_status);
+    e = launch_chained(select_topk_kernel<false>, dim3(s.batch), dim3(kThreads), fixed, stream, s, scores, cu_seqlens, keep_counts,
+                       protect, q_idx, cu_qlens, keep_idx, cu_keep, reinterpret_cast<unsigned*>(ws + w.keys_off), device_status);
   }
   count_launches(1);
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 // ---- fastav_select_noalloc: the same selection with its scratch inside the library ----------
