@@ -18,7 +18,8 @@ namespace fastav {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kUnroll = 4;  // key rows in flight per lane group
+// Key rows in flight per lane group: more when fewer query rows occupy the registers.
+template <int ROWS> struct Unroll { static constexpr int value = ROWS == 4 ? 8 : 4; };
 
 __device__ __forceinline__ void unpack8(const uint4& v, float2 (&out)[4]) {
   out[0] = make_float2(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u));
@@ -30,11 +31,12 @@ __device__ __forceinline__ void unpack8(const uint4& v, float2 (&out)[4]) {
 // DIM: head_dim; ROWS: query rows handled per pass (4 or 8); HB: KV heads covered by one block.
 // A "lane group" is the DIM/8 lanes that together read one key row of one KV head.
 template <int DIM, int ROWS>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, ROWS == 4 ? 3 : 2)
 score_narrow_logits_kernel(Shapes s, const uint16_t* __restrict__ q, const int32_t* __restrict__ q_idx,
                            const int32_t* __restrict__ cu_qlens, const uint16_t* __restrict__ k,
                            const int32_t* __restrict__ cu_seqlens, float* __restrict__ logits, int rq, int heads_per_block,
                            int chunk_keys) {
+  constexpr int kUnroll = Unroll<ROWS>::value;
   constexpr int kLanes = DIM / 8;               // lanes per key row
   constexpr int kGroups = kThreads / kLanes;    // key rows per block per step
   constexpr int kHalvings = ROWS == 8 ? 3 : 2;  // butterfly steps that halve the row set
@@ -141,36 +143,50 @@ __global__ void __launch_bounds__(256) score_narrow_stats_kernel(Shapes s, const
   const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
   const float* z = logits + ((long long)head * rq + r) * s.total_tokens + tok0;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  float m = -INFINITY;
-  for (int j = threadIdx.x; j < n; j += 256) m = fmaxf(m, z[j]);
+  // One pass: every thread keeps a running (max, sum 2^(z - max)) over its strided share, four loads at a time.
+  float m = -INFINITY, l = 0.f;
+  for (int j0 = threadIdx.x; j0 < n; j0 += 256 * 4) {
+    float v[4];
 #pragma unroll
-  for (int d = 16; d; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, d));
-  if (lane == 0) red[warp] = m;
+    for (int u = 0; u < 4; ++u) v[u] = j0 + u * 256 < n ? z[j0 + u * 256] : -INFINITY;
+    const float m_new = fmaxf(fmaxf(m, fmaxf(v[0], v[1])), fmaxf(v[2], v[3]));
+    if (m_new > -INFINITY) {
+      l = l * exp2f(m - m_new);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) l += exp2f(v[u] - m_new);
+      m = m_new;
+    }
+  }
+  // Merge the per-thread pairs: first the maximum, then the rescaled sums, both in a fixed order.
+  float bm = m;
+#pragma unroll
+  for (int d = 16; d; d >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xFFFFFFFFu, bm, d));
+  if (lane == 0) red[warp] = bm;
   __syncthreads();
-  m = red[0];
+  bm = red[0];
 #pragma unroll
-  for (int w = 1; w < 8; ++w) m = fmaxf(m, red[w]);
+  for (int w = 1; w < 8; ++w) bm = fmaxf(bm, red[w]);
   __syncthreads();
-  float l = 0.f;
-  if (m > -INFINITY)
-    for (int j = threadIdx.x; j < n; j += 256) l += exp2f(z[j] - m);
+  float part = (m > -INFINITY) ? l * exp2f(m - bm) : 0.f;
 #pragma unroll
-  for (int d = 16; d; d >>= 1) l += __shfl_xor_sync(0xFFFFFFFFu, l, d);
-  if (lane == 0) red[warp] = l;
+  for (int d = 16; d; d >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, d);
+  if (lane == 0) red[warp] = part;
   __syncthreads();
   if (threadIdx.x == 0) {
     float total = 0.f;
 #pragma unroll
     for (int w = 0; w < 8; ++w) total += red[w];
-    lse[(long long)(row0 + r) * s.hq + head] = total > 0.f ? m + log2f(total) : INFINITY;  // a row that sees no key adds 0
+    lse[(long long)(row0 + r) * s.hq + head] = total > 0.f ? bm + log2f(total) : INFINITY;  // a row that sees no key adds 0
   }
 }
 
-__global__ void __launch_bounds__(256) score_narrow_finalize_kernel(Shapes s, const int32_t* __restrict__ cu_qlens,
-                                                                    const int32_t* __restrict__ cu_seqlens,
-                                                                    const float* __restrict__ logits, int rq,
-                                                                    const float* __restrict__ lse,
-                                                                    float* __restrict__ scores) {
+constexpr int kFinalizeThreads = 64;  // small blocks: a few thousand tokens still spread over all SMs
+
+__global__ void __launch_bounds__(kFinalizeThreads) score_narrow_finalize_kernel(Shapes s, const int32_t* __restrict__ cu_qlens,
+                                                                                 const int32_t* __restrict__ cu_seqlens,
+                                                                                 const float* __restrict__ logits, int rq,
+                                                                                 const float* __restrict__ lse,
+                                                                                 float* __restrict__ scores) {
   extern __shared__ float lse_sh[];  // [Hq][rows]
   pdl_trigger();
   pdl_wait();
@@ -178,19 +194,28 @@ __global__ void __launch_bounds__(256) score_narrow_finalize_kernel(Shapes s, co
   const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
   if ((int)(blockIdx.x * blockDim.x) >= n) return;
   const int row0 = cu_qlens[b], all_rows = cu_qlens[b + 1] - row0, rows = min(all_rows, rq);
-  for (int i = threadIdx.x; i < s.hq * rows; i += blockDim.x) {
+  const int terms = s.hq * rows;
+  for (int i = threadIdx.x; i < terms; i += blockDim.x) {
     const int head = i / rows, r = i % rows;
     lse_sh[i] = lse[(long long)(row0 + r) * s.hq + head];
   }
   __syncthreads();
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   if (j >= n) return;
+  // Term i = (head, row) in head-major order; eight loads in flight, one running sum in that fixed order.
+  const float* z = logits + tok0 + j;
   float total = 0.f;
-  for (int head = 0; head < s.hq; ++head)
-    for (int r = 0; r < rows; ++r) {
-      const float z = logits[((long long)head * rq + r) * s.total_tokens + tok0 + j];
-      total += exp2f(z - lse_sh[head * rows + r]);
+  for (int i0 = 0; i0 < terms; i0 += 8) {
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = i0 + u;
+      v[u] = i < terms ? z[((long long)(i / rows) * rq + i % rows) * s.total_tokens] : -INFINITY;
     }
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      if (i0 + u < terms) total += exp2f(v[u] - lse_sh[i0 + u]);
+  }
   scores[tok0 + j] = all_rows > 0 ? total / ((float)s.hq * (float)all_rows) : 0.f;
 }
 
@@ -202,7 +227,7 @@ cudaError_t launch_logits(const Shapes& s, const uint16_t* q, const int32_t* q_i
   int hb = 1;
   while (hb * 2 <= s.hkv && s.hkv % (hb * 2) == 0 && hb * 2 <= kGroups) hb *= 2;
   const int keys_per_step = kGroups / hb;
-  const int quantum = keys_per_step * kUnroll;
+  const int quantum = keys_per_step * Unroll<ROWS>::value;
   // Enough blocks to fill the machine a few times over, but never less than one unrolled step each.
   const long long want_blocks = (long long)kNumSMs * 8;
   long long chunk = ((long long)s.total_tokens * (s.hkv / hb) + want_blocks - 1) / want_blocks;
@@ -239,7 +264,8 @@ cudaError_t launch_score_narrow(const Shapes& s, const Workspace& w, const void*
   if ((e = launch_chained(score_narrow_stats_kernel, dim3(s.hq * rq, s.batch), dim3(256), 0, stream, s, cu_qlens, cu_seqlens,
                           (const float*)logits, rq, lse)) != cudaSuccess)
     return e;
-  if ((e = launch_chained(score_narrow_finalize_kernel, dim3((s.max_seqlen + 255) / 256, s.batch), dim3(256),
+  if ((e = launch_chained(score_narrow_finalize_kernel, dim3((s.max_seqlen + kFinalizeThreads - 1) / kFinalizeThreads, s.batch),
+                          dim3(kFinalizeThreads),
                           s.hq * rq * sizeof(float), stream, s, cu_qlens, cu_seqlens, (const float*)logits, rq, (const float*)lse,
                           scores_out)) != cudaSuccess)
     return e;

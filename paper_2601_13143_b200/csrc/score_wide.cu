@@ -615,23 +615,36 @@ __global__ void __launch_bounds__(256) score_wide_merge_kernel(Shapes s, const i
   if (lane == 0) lse[w] = (l > 0.f) ? m + log2f(l) : INFINITY;  // a row that sees no key contributes 0
 }
 
-__global__ void __launch_bounds__(256) score_wide_finalize_kernel(Shapes s, const int32_t* __restrict__ cu_seqlens,
-                                                                  const int32_t* __restrict__ cu_qlens, int rc_max,
-                                                                  int rows_per_chunk, const float* __restrict__ partial,
-                                                                  float* __restrict__ scores) {
+constexpr int kFinalizeThreads = 64;
+
+__global__ void __launch_bounds__(kFinalizeThreads) score_wide_finalize_kernel(Shapes s, const int32_t* __restrict__ cu_seqlens,
+                                                                               const int32_t* __restrict__ cu_qlens, int rc_max,
+                                                                               int rows_per_chunk, const float* __restrict__ partial,
+                                                                               float* __restrict__ scores) {
   pdl_trigger();
   const int b = blockIdx.y;
   const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
   const int rows = cu_qlens[b + 1] - cu_qlens[b];
   const int row_chunks = (rows * s.group + rows_per_chunk - 1) / rows_per_chunk;
-  pdl_wait();
   const float inv = rows > 0 ? 1.0f / ((float)s.hq * (float)rows) : 0.f;
-  for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < n; j += gridDim.x * blockDim.x) {
-    float total = 0.f;
-    for (int g = 0; g < s.hkv; ++g)
-      for (int rc = 0; rc < row_chunks; ++rc) total += partial[(long long)(g * rc_max + rc) * s.total_tokens + tok0 + j];
-    scores[tok0 + j] = total * inv;
+  pdl_wait();
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= n) return;
+  // Partial i = (KV head, row chunk) in that order; eight loads in flight, one running sum in fixed order.
+  const int terms = s.hkv * row_chunks;
+  const float* col = partial + tok0 + j;
+  float total = 0.f;
+  for (int i0 = 0; i0 < terms; i0 += 8) {
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = i0 + u;
+      v[u] = i < terms ? col[(long long)((i / row_chunks) * rc_max + i % row_chunks) * s.total_tokens] : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) total += v[u];
   }
+  scores[tok0 + j] = total * inv;
 }
 
 // ---- host side -----------------------------------------------------------------------------------
@@ -704,7 +717,8 @@ cudaError_t run(const Shapes& s, const Workspace& w, const CUtensorMap& k_map, c
                           cu_seqlens, (int)chunk_tiles, stat_chunks, rc_max, rows_per_chunk, (float2*)nullptr, (const float*)lse,
                           partial, device_status)) != cudaSuccess)
     return e;
-  if ((e = launch_chained(score_wide_finalize_kernel, dim3((s.max_seqlen + 255) / 256, s.batch), dim3(256), 0, stream, s,
+  if ((e = launch_chained(score_wide_finalize_kernel, dim3((s.max_seqlen + kFinalizeThreads - 1) / kFinalizeThreads, s.batch),
+                          dim3(kFinalizeThreads), 0, stream, s,
                           cu_seqlens, cu_qlens, rc_max, rows_per_chunk, (const float*)partial, scores_out)) != cudaSuccess)
     return e;
   count_launches(4);

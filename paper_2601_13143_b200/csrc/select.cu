@@ -2,8 +2,11 @@
 //
 // One thread block per sequence.  Scores become order-preserving 32-bit keys (protected tokens get
 // the largest key), held in shared memory when the sequence fits.  The k-th largest key T is found
-// by an MSB-first radix select (4 passes of 8 bits, shared-memory histograms fed by warp-aggregated
-// atomics).  A block-wide prefix scan in index order then keeps every key above T plus the first
+// by an MSB-first radix select over the bits in which the keys of the sequence actually differ
+// (the common leading bits come from a min/max reduction; softmax scores share most of their
+// exponent, so without this the first histogram would pile into a handful of bins): at most three
+// passes of 11-bit digits, shared-memory histograms, a block-wide suffix scan to pick the bin.
+// A single blocked prefix scan in index order then keeps every key above T plus the first
 // (k - #above) keys equal to T: ties go to the lower index and survivors come out ascending, which
 // is exactly the order the gather that follows needs.  Integer work throughout: the result is a
 // unique function of the fp32 score bits.
@@ -16,6 +19,8 @@ namespace {
 
 constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
+constexpr int kDigitBits = 11;
+constexpr int kBins = 1 << kDigitBits;
 constexpr unsigned kProtectedKey = 0xFFFFFFFFu;
 
 // fp32 -> uint32 with the same ordering as the float comparison (-0 and +0 compare equal).
@@ -26,13 +31,19 @@ __device__ __forceinline__ unsigned order_key(float x) {
 }
 
 struct SelectShared {
-  unsigned hist[256];
-  unsigned warp_totals[2][kWarps];
+  unsigned hist[kBins];
+  unsigned warp_a[kWarps], warp_b[kWarps];
+  unsigned key_min, key_max;
   unsigned prefix;      // bits of T fixed so far
   int remaining;        // how many more keys (from the top of the current bucket) are still to take
   int base;             // output offset of this sequence
   int protected_count;
 };
+
+// Shared-memory slot of key j: one word of padding per 32 keeps both the strided and the blocked
+// access patterns below (nearly) free of bank conflicts.
+template <bool kKeysInShared>
+__device__ __forceinline__ int slot(int j) { return kKeysInShared ? j + (j >> 5) : j; }
 
 template <bool kKeysInShared>
 __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const float* __restrict__ scores,
@@ -48,13 +59,12 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
   unsigned* keys = kKeysInShared ? reinterpret_cast<unsigned*>(smem_raw + sizeof(SelectShared)) : nullptr;
 
   pdl_trigger();
-  pdl_wait();  // the scores are the previous kernel's output
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
   if (!kKeysInShared) keys = keys_global + tok0;
 
   // Output offset: prefix sum of the clamped keep counts of the sequences before this one.
-  if (tid == 0) { sh.base = 0; sh.protected_count = 0; }
+  if (tid == 0) { sh.base = 0; sh.protected_count = 0; sh.key_min = 0xFFFFFFFFu; sh.key_max = 0u; }
   __syncthreads();
   {
     int part = 0;
@@ -71,109 +81,158 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
   int k = keep_counts[b];
   k = k < 0 ? 0 : (k > n ? n : k);
 
+  pdl_wait();  // the scores are the previous kernel's output
+
   // Keys.
-  for (int j = tid; j < n; j += kThreads) {
-    unsigned key = order_key(scores[tok0 + j]);
-    if (key == kProtectedKey) key = kProtectedKey - 1;  // only a NaN pattern lands here
-    if (protect && protect[tok0 + j]) key = kProtectedKey;
-    keys[j] = key;
+  for (int j0 = tid; j0 < n; j0 += kThreads * 8) {
+    float v[8];  // eight independent loads in flight per thread: one block serves a whole sequence
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int j = j0 + u * kThreads;
+      v[u] = j < n ? __ldg(scores + tok0 + j) : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int j = j0 + u * kThreads;
+      if (j < n) {
+        unsigned key = order_key(v[u]);
+        if (key == kProtectedKey) key = kProtectedKey - 1;  // only a NaN pattern lands here
+        if (protect && protect[tok0 + j]) key = kProtectedKey;
+        keys[slot<kKeysInShared>(j)] = key;
+      }
+    }
   }
   __syncthreads();
   if (s.flags & FASTAV_PROTECT_QUERY_ROWS) {
     for (int r = cu_qlens[b] + tid; r < cu_qlens[b + 1]; r += kThreads) {
       const int j = q_idx[r];
-      if (j >= 0 && j < n) keys[j] = kProtectedKey;
+      if (j >= 0 && j < n) keys[slot<kKeysInShared>(j)] = kProtectedKey;
     }
     __syncthreads();
   }
-  const int base = sh.base;
+  // Range of the unprotected keys and number of protected ones.
+  {
+    unsigned lo = 0xFFFFFFFFu, hi = 0u;
+    int prot = 0;
+    for (int j = tid; j < n; j += kThreads) {
+      const unsigned key = keys[slot<kKeysInShared>(j)];
+      if (key == kProtectedKey) ++prot;
+      else { lo = min(lo, key); hi = max(hi, key); }
+    }
+    lo = __reduce_min_sync(0xFFFFFFFFu, lo);
+    hi = __reduce_max_sync(0xFFFFFFFFu, hi);
+    prot = __reduce_add_sync(0xFFFFFFFFu, prot);
+    if (lane == 0) {
+      atomicMin(&sh.key_min, lo);
+      atomicMax(&sh.key_max, hi);
+      if (prot) atomicAdd(&sh.protected_count, prot);
+    }
+  }
+  __syncthreads();
+  const int base = sh.base, n_protected = sh.protected_count;
+  const unsigned key_min = sh.key_min, key_max = sh.key_max;
   if (tid == 0) {
     cu_keep[b + 1] = base + k;
     if (b == 0) cu_keep[0] = 0;
-    sh.prefix = 0;
-    sh.remaining = k;
+    if (n_protected > k && device_status) atomicOr(device_status, FASTAV_DEV_PROTECT_OVERFLOW);
   }
   if (k == 0 || n == 0) return;
 
-  // Radix select: after pass p the top 8(p+1) bits of T are known.
-  for (int pass = 0; pass < 4; ++pass) {
-    const int shift = 24 - 8 * pass;
-    for (int i = tid; i < 256; i += kThreads) sh.hist[i] = 0;
-    __syncthreads();
-    const unsigned prefix = sh.prefix;
-    const unsigned high_mask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
-    const int rounds = (n + kThreads - 1) / kThreads;
-    for (int rd = 0; rd < rounds; ++rd) {
-      const int j = rd * kThreads + tid;
-      const bool in_bucket = j < n && ((keys[j] & high_mask) == prefix);
-      const unsigned digit = in_bucket ? ((keys[j] >> shift) & 0xFFu) : 0x100u;
-      const unsigned peers = __match_any_sync(0xFFFFFFFFu, digit);
-      if (in_bucket && lane == (__ffs(peers) - 1)) atomicAdd(&sh.hist[digit], (unsigned)__popc(peers));
+  unsigned T;
+  int need_eq;  // how many keys equal to T are kept (the lowest-index ones)
+  if (k <= n_protected) {
+    T = kProtectedKey;  // protected tokens alone fill the keep set
+    need_eq = k;
+  } else if (key_min == key_max) {
+    T = key_min;  // every unprotected key is the same
+    need_eq = k - n_protected;
+  } else {
+    // Radix select of the (k - #protected)-th largest unprotected key over the bits below the common prefix.
+    int bits_left = 32 - __clz(key_min ^ key_max);  // >= 1
+    if (tid == 0) {
+      sh.prefix = bits_left == 32 ? 0u : (key_min >> bits_left) << bits_left;
+      sh.remaining = k - n_protected;
     }
-    __syncthreads();
-    if (warp == 0) {
-      // Walk the 256 bins from the top; lane l owns bins [8l, 8l+8).
-      unsigned local[8], sum = 0;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) { local[i] = sh.hist[lane * 8 + i]; sum += local[i]; }
-      unsigned above = sum;  // inclusive suffix sum over lanes (higher lanes = larger digits)
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        const unsigned t = __shfl_down_sync(0xFFFFFFFFu, above, d);
-        if (lane + d < 32) above += t;
-      }
-      const unsigned rem = (unsigned)sh.remaining;
-      const unsigned strictly_above = above - sum;  // keys in bins of higher lanes
-      if (strictly_above < rem && rem <= above) {   // the k-th key falls in one of this lane's bins
-        unsigned acc = strictly_above;
-        for (int i = 7; i >= 0; --i) {
-          if (acc + local[i] >= rem) {
-            sh.prefix = prefix | ((unsigned)(lane * 8 + i) << shift);
-            sh.remaining = (int)(rem - acc);
-            break;
-          }
-          acc += local[i];
+    while (bits_left > 0) {
+      const int width = min(kDigitBits, bits_left), shift = bits_left - width;
+      for (int i = tid; i < kBins; i += kThreads) sh.hist[i] = 0;
+      __syncthreads();
+      const unsigned prefix = sh.prefix;
+      const unsigned digit_mask = (1u << width) - 1u;
+      const int rounds = (n + kThreads - 1) / kThreads;
+      for (int rd = 0; rd < rounds; ++rd) {
+        const int j = rd * kThreads + tid;
+        const unsigned key = j < n ? keys[slot<kKeysInShared>(j)] : kProtectedKey;
+        // in the bucket: unprotected and equal to the prefix in the bits above this digit
+        const bool in_bucket = key != kProtectedKey && (bits_left == 32 || (key >> bits_left) == (prefix >> bits_left));
+        const unsigned digit = in_bucket ? ((key >> shift) & digit_mask) : 0xFFFFu;
+        int same;
+        __match_all_sync(0xFFFFFFFFu, digit, &same);
+        if (same) {  // a run of equal scores (typically zeros): one add for the warp
+          if (in_bucket && lane == 0) atomicAdd(&sh.hist[digit], 32u);
+        } else if (in_bucket) {
+          atomicAdd(&sh.hist[digit], 1u);
         }
       }
-    }
-    __syncthreads();
-  }
-  const unsigned T = sh.prefix;
-  const int need_eq = sh.remaining;  // how many keys equal to T are kept (the lowest-index ones)
-
-  // Stable compaction in index order.
-  int run_gt = 0, run_eq = 0;
-  const bool global_idx = (s.flags & FASTAV_KEEP_IDX_GLOBAL) != 0;
-  const int rounds = (n + kThreads - 1) / kThreads;
-  for (int rd = 0; rd < rounds; ++rd) {
-    const int j = rd * kThreads + tid;
-    const unsigned key = j < n ? keys[j] : 0u;
-    const bool gt = j < n && key > T, eq = j < n && key == T;
-    const unsigned m_gt = __ballot_sync(0xFFFFFFFFu, gt), m_eq = __ballot_sync(0xFFFFFFFFu, eq);
-    const unsigned lt_mask = (1u << lane) - 1u;
-    unsigned* totals = sh.warp_totals[rd & 1];
-    if (lane == 0) totals[warp] = (unsigned)__popc(m_gt) | ((unsigned)__popc(m_eq) << 16);
-    __syncthreads();
-    unsigned incl = totals[lane];  // packed (gt, eq) counts never exceed 1024 per round: no carry between halves
+      __syncthreads();
+      // Suffix sums over the bins, two bins per thread, to find the bin holding the wanted key.
+      const unsigned h0 = sh.hist[2 * tid], h1 = sh.hist[2 * tid + 1];
+      unsigned incl = h0 + h1;  // inclusive suffix sum over threads (higher threads = larger digits)
 #pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-      const unsigned t = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-      if (lane >= d) incl += t;
+      for (int d = 1; d < 32; d <<= 1) {
+        const unsigned t = __shfl_down_sync(0xFFFFFFFFu, incl, d);
+        if (lane + d < 32) incl += t;
+      }
+      if (lane == 0) sh.warp_a[warp] = incl;
+      __syncthreads();
+      unsigned above_warp = 0;
+      for (int w = warp + 1; w < kWarps; ++w) above_warp += sh.warp_a[w];
+      const unsigned above_me = above_warp + incl - (h0 + h1);  // keys in bins above this thread's two
+      const unsigned rem = (unsigned)sh.remaining;
+      __syncthreads();  // everyone has read `remaining` before the one owner rewrites it
+      if (above_me < rem && rem <= above_me + h0 + h1) {
+        const bool upper = rem <= above_me + h1;
+        const unsigned bin = 2 * tid + (upper ? 1 : 0);
+        sh.prefix = prefix | (bin << shift);
+        sh.remaining = (int)(rem - above_me - (upper ? 0u : h1));
+      }
+      __syncthreads();
+      bits_left = shift;
     }
-    const unsigned round_total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-    const unsigned before_warp = warp == 0 ? 0u : __shfl_sync(0xFFFFFFFFu, incl, warp - 1);
-    const int gt_before = run_gt + (int)(before_warp & 0xFFFFu) + __popc(m_gt & lt_mask);
-    const int eq_before = run_eq + (int)(before_warp >> 16) + __popc(m_eq & lt_mask);
-    if (gt || (eq && eq_before < need_eq)) {
-      const int out = gt_before + (eq_before < need_eq ? eq_before : need_eq);
+    T = sh.prefix;
+    need_eq = sh.remaining;
+  }
+
+  // Stable compaction in index order: thread t owns the `per` consecutive tokens starting at t * per.
+  const bool global_idx = (s.flags & FASTAV_KEEP_IDX_GLOBAL) != 0;
+  const int per = (n + kThreads - 1) / kThreads;
+  const int j0 = tid * per, j1 = min(n, j0 + per);
+  unsigned my_gt = 0, my_eq = 0;
+  for (int j = j0; j < j1; ++j) {
+    const unsigned key = keys[slot<kKeysInShared>(j)];
+    my_gt += key > T;
+    my_eq += key == T;
+  }
+  unsigned gt_incl = my_gt, eq_incl = my_eq;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const unsigned a = __shfl_up_sync(0xFFFFFFFFu, gt_incl, d), c = __shfl_up_sync(0xFFFFFFFFu, eq_incl, d);
+    if (lane >= d) { gt_incl += a; eq_incl += c; }
+  }
+  if (lane == 31) { sh.warp_a[warp] = gt_incl; sh.warp_b[warp] = eq_incl; }
+  __syncthreads();
+  unsigned gt_before = gt_incl - my_gt, eq_before = eq_incl - my_eq;
+  for (int w = 0; w < warp; ++w) { gt_before += sh.warp_a[w]; eq_before += sh.warp_b[w]; }
+  for (int j = j0; j < j1; ++j) {
+    const unsigned key = keys[slot<kKeysInShared>(j)];
+    const bool gt = key > T, eq = key == T;
+    if (gt || (eq && (int)eq_before < need_eq)) {
+      const int out = (int)gt_before + min((int)eq_before, need_eq);
       keep_idx[base + out] = global_idx ? tok0 + j : j;
     }
-    if (key == kProtectedKey && j < n) atomicAdd(&sh.protected_count, 1);
-    run_gt += (int)(round_total & 0xFFFFu);
-    run_eq += (int)(round_total >> 16);
+    gt_before += gt;
+    eq_before += eq;
   }
-  __syncthreads();
-  if (tid == 0 && sh.protected_count > k && device_status) atomicOr(device_status, FASTAV_DEV_PROTECT_OVERFLOW);
 }
 
 }  // namespace
@@ -183,7 +242,7 @@ cudaError_t launch_select(const Shapes& s, const Workspace& w, const float* scor
                           const int32_t* cu_qlens, int32_t* keep_idx, int32_t* cu_keep, unsigned char* ws,
                           int32_t* device_status, cudaStream_t stream) {
   const size_t fixed = sizeof(SelectShared);
-  const size_t want = fixed + (size_t)s.max_seqlen * sizeof(unsigned);
+  const size_t want = fixed + ((size_t)s.max_seqlen + s.max_seqlen / 32 + 1) * sizeof(unsigned);
   constexpr size_t kMaxDynamic = 227 * 1024 - 1024;
   cudaError_t e;
   if (want <= kMaxDynamic) {
