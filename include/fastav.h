@@ -60,6 +60,10 @@ extern "C" {
 #define FASTAV_SCORE_PATH_WIDE 0x300u    /* tensor-core path */
 #define FASTAV_SCORE_PATH_MASK 0x300u
 
+/* Diagnostics: make fastav_compact use its plain load/store kernel instead of the bulk-copy one. */
+#define FASTAV_COMPACT_PATH_LOADSTORE 0x400u
+#define FASTAV_COMPACT_PATH_MASK 0x400u
+
 /* bits OR-ed into *device_status */
 #define FASTAV_DEV_K_CLAMPED 1        /* some keep_counts[b] was outside [0, n_b] and was clamped */
 #define FASTAV_DEV_PROTECT_OVERFLOW 2 /* more protected tokens than k_b: the lowest-index ones were kept */

@@ -87,6 +87,10 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a -
 #ifdef __CUDACC__
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// A pointer to data the predecessor writes must be passed through this after pdl_wait: the compiler
+// may otherwise hoist loads through a `const __restrict__` pointer above the wait (it is entitled to
+// assume nobody writes such data while the kernel runs).
+#define pdl_acquire(ptr) asm volatile("" : "+l"(ptr) : : "memory")
 
 template <typename... KArgs, typename... Args>
 cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {

@@ -44,6 +44,8 @@ score_narrow_logits_kernel(Shapes s, const uint16_t* __restrict__ q, const int32
 
   pdl_trigger();
   pdl_wait();  // q and k may be what the previous kernel wrote; the logits may still be read by it
+  pdl_acquire(q);
+  pdl_acquire(k);
   const int b = blockIdx.z;
   const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
   const int key_begin = blockIdx.x * chunk_keys;
@@ -137,6 +139,7 @@ __global__ void __launch_bounds__(256) score_narrow_stats_kernel(Shapes s, const
   __shared__ float red[8];
   pdl_trigger();
   pdl_wait();
+  pdl_acquire(logits);
   const int b = blockIdx.y, head = blockIdx.x / rq, r = blockIdx.x % rq;
   const int row0 = cu_qlens[b], rows = min(cu_qlens[b + 1] - row0, rq);
   if (r >= rows) return;
@@ -190,6 +193,8 @@ __global__ void __launch_bounds__(kFinalizeThreads) score_narrow_finalize_kernel
   extern __shared__ float lse_sh[];  // [Hq][rows]
   pdl_trigger();
   pdl_wait();
+  pdl_acquire(logits);
+  pdl_acquire(lse);
   const int b = blockIdx.y;
   const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
   if ((int)(blockIdx.x * blockDim.x) >= n) return;

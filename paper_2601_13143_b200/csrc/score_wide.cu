@@ -466,6 +466,7 @@ score_wide_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
     const int my_lane = quarter * 32 + lane;  // row (sweep 1) or key (sweep 2) inside the tile
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
     pdl_wait();  // before the first read of lse (sweep 2) and the first write of stats / partial
+    pdl_acquire(lse);
 
     if constexpr (SWEEP == 1) {
       // Warpgroup (e, h) owns the rows of 128-row tile e and the keys [64 h, 64 h + 64) of every K tile:
@@ -589,6 +590,7 @@ __global__ void __launch_bounds__(256) score_wide_merge_kernel(Shapes s, const i
                                                                int chunk_keys, float* __restrict__ lse) {
   pdl_trigger();
   pdl_wait();
+  pdl_acquire(stats);
   const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (w >= s.total_q * s.hq) return;
   const int row = w / s.hq;
@@ -628,6 +630,7 @@ __global__ void __launch_bounds__(kFinalizeThreads) score_wide_finalize_kernel(S
   const int row_chunks = (rows * s.group + rows_per_chunk - 1) / rows_per_chunk;
   const float inv = rows > 0 ? 1.0f / ((float)s.hq * (float)rows) : 0.f;
   pdl_wait();
+  pdl_acquire(partial);
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   if (j >= n) return;
   // Partial i = (KV head, row chunk) in that order; eight loads in flight, one running sum in fixed order.

@@ -82,6 +82,7 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
   k = k < 0 ? 0 : (k > n ? n : k);
 
   pdl_wait();  // the scores are the previous kernel's output
+  pdl_acquire(scores);
 
   // Keys.
   for (int j0 = tid; j0 < n; j0 += kThreads * 8) {

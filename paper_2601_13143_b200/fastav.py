@@ -20,6 +20,7 @@ FASTAV_KEEP_IDX_GLOBAL = 4
 FASTAV_SCORE_PATH_GENERIC = 0x100
 FASTAV_SCORE_PATH_NARROW = 0x200
 FASTAV_SCORE_PATH_WIDE = 0x300
+FASTAV_COMPACT_PATH_LOADSTORE = 0x400
 
 FASTAV_DEV_K_CLAMPED = 1
 FASTAV_DEV_PROTECT_OVERFLOW = 2

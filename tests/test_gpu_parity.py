@@ -192,7 +192,8 @@ def test_select_sequence_longer_than_shared_memory():
 # ---- compact ----------------------------------------------------------------------------------
 
 @pytest.mark.parametrize("hkv,d,hid", [(2, 64, 64), (4, 128, 3584), (8, 128, 4096), (1, 64, 8)])
-def test_compact_matches_oracle(hkv, d, hid):
+@pytest.mark.parametrize("path", [0, fastav.FASTAV_COMPACT_PATH_LOADSTORE])
+def test_compact_matches_oracle(hkv, d, hid, path):
     rng = np.random.default_rng(hkv * 100 + d)
     lens = [37, 0, 129, 1]
     keeps = [10, 0, 129, 1]
@@ -202,7 +203,7 @@ def test_compact_matches_oracle(hkv, d, hid):
     keep_idx = np.concatenate([np.sort(rng.choice(n, size=k, replace=False)) for n, k in zip(lens, keeps)]).astype(np.int32)
     cu_keep = np.concatenate([[0], np.cumsum(keeps)]).astype(np.int32)
     ref = oracle.compact(keep_idx, cu_keep, cu, bf16_bits(p.hidden), p.pos.numpy(), bf16_bits(p.k), bf16_bits(p.v))
-    buf = parity.to_device(p, flags=0)
+    buf = parity.to_device(p, flags=path)
     for t in (buf.hidden_out, buf.k_out, buf.v_out):
         t.view(torch.int16).fill_(0x7FC1)
     buf.pos_out.fill_(-1)
@@ -213,13 +214,42 @@ def test_compact_matches_oracle(hkv, d, hid):
     for name in ("hidden", "pos", "k", "v"):
         parity.assert_bits_equal(getattr(buf, name + "_out"), ref[name], name)
     # global indices, only the K pair
-    buf.params.flags = fastav.FASTAV_KEEP_IDX_GLOBAL
+    buf.params.flags = fastav.FASTAV_KEEP_IDX_GLOBAL | path
     global_idx = np.concatenate([cu[b] + keep_idx[cu_keep[b]:cu_keep[b + 1]] for b in range(len(lens))]).astype(np.int32)
     buf.keep_idx[:len(global_idx)].copy_(torch.as_tensor(global_idx))
     buf.k_out.zero_()
     fastav.fastav_compact(buf.params, buf.keep_idx, buf.cu_keep, buf.cu_seqlens, k_in=buf.k, k_out=buf.k_out)
     torch.cuda.synchronize()
     parity.assert_bits_equal(buf.k_out, ref["k"], "k (global indices)")
+
+
+def test_compact_many_rows_per_warp_and_bad_rows_in_between():
+    """Enough rows that every warp of the bulk-copy kernel cycles its slots many times, with a few
+    out-of-range indices sprinkled in (skipped rows must not disturb the rows around them)."""
+    rng = np.random.default_rng(77)
+    lens, keeps = [9000, 3000], [7000, 3000]
+    p = W.random_problem(seed=5, lens=lens, rows=[1, 1], keeps=keeps, num_q_heads=4, num_kv_heads=2, head_dim=64, hidden=256)
+    cu = p.cu_seqlens.numpy()
+    keep_idx = np.concatenate([np.sort(rng.choice(n, size=k, replace=False)) for n, k in zip(lens, keeps)]).astype(np.int32)
+    cu_keep = np.concatenate([[0], np.cumsum(keeps)]).astype(np.int32)
+    ref = oracle.compact(keep_idx, cu_keep, cu, bf16_bits(p.hidden), p.pos.numpy(), bf16_bits(p.k), bf16_bits(p.v))
+    bad_rows = [5, 1234, 6999, 7000, 9999]
+    broken = keep_idx.copy()
+    broken[bad_rows] = [-1, 9000, 20000, 3000, -5]
+    buf = parity.to_device(p, flags=0)
+    for t in (buf.hidden_out, buf.k_out, buf.v_out):
+        t.view(torch.int16).fill_(0x7FC1)
+    buf.keep_idx[:len(broken)].copy_(torch.as_tensor(broken))
+    buf.cu_keep.copy_(torch.as_tensor(cu_keep))
+    buf.compact()
+    assert _sync_status(buf) == fastav.FASTAV_DEV_BAD_INDEX
+    good = np.ones(len(keep_idx), dtype=bool)
+    good[bad_rows] = False
+    for name in ("hidden", "k", "v"):
+        got = getattr(buf, name + "_out").cpu().view(torch.int16).numpy()
+        want = ref[name].view(np.int16)
+        assert np.array_equal(got[good], want[good]), name
+        assert (got[~good] == 0x7FC1).all(), name + ": a skipped row was written"
 
 
 def test_compact_strided_outputs_and_guard_bands():
