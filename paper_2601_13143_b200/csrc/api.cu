@@ -166,7 +166,7 @@ cudaError_t launch_score(const Shapes& s, const Workspace& w, const void* q, con
   const unsigned forced = s.flags & FASTAV_SCORE_PATH_MASK;
   if (forced == FASTAV_SCORE_PATH_GENERIC) return launch_score_generic(s, w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out, ws, stream);
   if (score_narrow_applies(s) && (forced == 0 || forced == FASTAV_SCORE_PATH_NARROW))
-    return launch_score_narrow(s, w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out, ws, stream);
+    return launch_score_narrow(s, w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out, ws, device_status, stream);
   if (score_wide_applies(s)) {
     bool used = false;
     const cudaError_t e = launch_score_wide(s, w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out, ws, device_status, stream, &used);

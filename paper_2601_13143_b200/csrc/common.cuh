@@ -50,7 +50,7 @@ constexpr int kNarrowMaxRows = 4;
 bool score_narrow_applies(const Shapes& s);
 cudaError_t launch_score_narrow(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
                                 const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
-                                unsigned char* ws, cudaStream_t stream);
+                                unsigned char* ws, int32_t* device_status, cudaStream_t stream);
 
 // Many scored rows per sequence: tensor-core path (tcgen05 + TMA).  `*used` is false when the TMA
 // descriptor for K could not be built; nothing was launched then and the caller takes another path.

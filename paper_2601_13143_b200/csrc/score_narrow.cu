@@ -2,8 +2,9 @@
 // itself uses in the fine-pruning stage: Q_last is one row per head, so Q K^T is a matrix-vector
 // product and the step is bound by reading K once from HBM.
 //
-//   logits   : every 16-byte piece of a key row is loaded once by one lane and multiplied with up to
-//              eight query rows held in registers (the rows and heads of one KV group); a butterfly
+//   logits   : K streams through a ring of shared-memory slots filled by bulk asynchronous copies; every
+//              16-byte piece of a key row is read once by one lane and multiplied with up to eight query
+//              rows held in registers (the rows and heads of one KV group); a butterfly
 //              of shuffles that halves the row set at each step leaves one finished logit per lane.
 //              Logits [Hq, R, N] (base-2 units, -inf where the causal mask hides the key) go to the
 //              workspace: R * Hq * 4 bytes per token next to the Hkv * d * 2 bytes of K read.
@@ -13,13 +14,15 @@
 // Every key goes through the same arithmetic in the same order, whatever its position, so equal
 // keys get bit-equal scores and runs are bit-reproducible.
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace fastav {
 namespace {
 
-constexpr int kThreads = 256;
-// Key rows in flight per lane group: more when fewer query rows occupy the registers.
-template <int ROWS> struct Unroll { static constexpr int value = ROWS == 4 ? 8 : 4; };
+constexpr int kComputeThreads = 256;             // 8 warps that multiply
+constexpr int kThreads = kComputeThreads + 32;   // + 1 warp that issues the copies
+constexpr int kStages = 3;                       // K slots in flight per block
+constexpr int kSlotKeys = 16;                    // tokens per slot
 
 __device__ __forceinline__ void unpack8(const uint4& v, float2 (&out)[4]) {
   out[0] = make_float2(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u));
@@ -28,21 +31,43 @@ __device__ __forceinline__ void unpack8(const uint4& v, float2 (&out)[4]) {
   out[3] = make_float2(__uint_as_float(v.w << 16), __uint_as_float(v.w & 0xFFFF0000u));
 }
 
-// DIM: head_dim; ROWS: query rows handled per pass (4 or 8); HB: KV heads covered by one block.
-// A "lane group" is the DIM/8 lanes that together read one key row of one KV head.
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst_smem),
+               "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
+// DIM: head_dim; ROWS: query rows handled per pass (4 or 8).  One block covers `heads_per_block` KV heads
+// of a chunk of keys.  A producer warp streams the K rows of those heads, 16 tokens per slot, into a ring
+// of shared-memory slots with bulk asynchronous copies; eight warps multiply.  A "lane group" is the DIM/8
+// lanes that together read one key row of one KV head; its query rows stay in registers.
 template <int DIM, int ROWS>
-__global__ void __launch_bounds__(kThreads, ROWS == 4 ? 3 : 2)
+__global__ void __launch_bounds__(kThreads, ROWS == 8 ? 1 : 2)
 score_narrow_logits_kernel(Shapes s, const uint16_t* __restrict__ q, const int32_t* __restrict__ q_idx,
                            const int32_t* __restrict__ cu_qlens, const uint16_t* __restrict__ k,
                            const int32_t* __restrict__ cu_seqlens, float* __restrict__ logits, int rq, int heads_per_block,
-                           int chunk_keys) {
-  constexpr int kUnroll = Unroll<ROWS>::value;
-  constexpr int kLanes = DIM / 8;               // lanes per key row
-  constexpr int kGroups = kThreads / kLanes;    // key rows per block per step
-  constexpr int kHalvings = ROWS == 8 ? 3 : 2;  // butterfly steps that halve the row set
+                           int chunk_keys, int32_t* device_status) {
+  constexpr int kLanes = DIM / 8;                     // lanes per key row
+  constexpr int kGroups = kComputeThreads / kLanes;   // key rows per block per step
+  constexpr int kHalvings = ROWS == 8 ? 3 : 2;        // butterfly steps that halve the row set
   constexpr int kPlainBits = (kLanes == 16 ? 4 : 3) - kHalvings;
+  extern __shared__ __align__(128) unsigned char ring_smem[];
+  __shared__ uint64_t full[kStages], empty[kStages];
+  __shared__ int abort_flag;
 
   pdl_trigger();
+  const int warp = threadIdx.x >> 5;
+  const int row_bytes = heads_per_block * DIM * 2;  // bytes of one token in a slot
+  const int slot_bytes = kSlotKeys * row_bytes;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kStages; ++i) {
+      ptx::mbar_init(ptx::smem_u32(&full[i]), 1);
+      ptx::mbar_init(ptx::smem_u32(&empty[i]), kComputeThreads / 32);
+    }
+    abort_flag = 0;
+    ptx::fence_barrier_init();
+  }
+  __syncthreads();
   pdl_wait();  // q and k may be what the previous kernel wrote; the logits may still be read by it
   pdl_acquire(q);
   pdl_acquire(k);
@@ -54,17 +79,50 @@ score_narrow_logits_kernel(Shapes s, const uint16_t* __restrict__ q, const int32
   const int row0 = cu_qlens[b], rows = min(cu_qlens[b + 1] - row0, rq);
   const int flat_rows = rows * s.group;
   if (flat_rows == 0) return;
+  const int passes = (flat_rows + ROWS - 1) / ROWS;
+  const int slots = (key_end - key_begin + kSlotKeys - 1) / kSlotKeys;  // per pass
+  const int head0 = blockIdx.y * heads_per_block;
+  const uint32_t ring = ptx::smem_u32(ring_smem);
 
+  if (warp == kComputeThreads / 32) {
+    // ---- producer: slot `it` (over all passes) holds tokens [key, key + 16) x heads [head0, head0 + hb) -------
+    const int lane = threadIdx.x & 31;
+    const bool packed = s.k_sh == DIM;  // the heads of a token are contiguous
+    const int pieces_per_token = packed ? 1 : heads_per_block;
+    const uint32_t piece_bytes = packed ? row_bytes : DIM * 2;
+    bool ok = true;
+    for (int it = 0; it < passes * slots && ok; ++it) {
+      const int stage = it % kStages;
+      ok = ptx::mbar_wait_bounded(ptx::smem_u32(&empty[stage]), ((it / kStages) & 1) ^ 1u, &abort_flag);
+      if (!ok) break;
+      const int key = key_begin + (it % slots) * kSlotKeys;
+      const int tokens = min(kSlotKeys, key_end - key);
+      const uint32_t bar = ptx::smem_u32(&full[stage]);
+      if (lane == 0) ptx::mbar_arrive_expect_tx(bar, tokens * row_bytes);
+      __syncwarp();
+      for (int piece = lane; piece < tokens * pieces_per_token; piece += 32) {
+        const int t = piece / pieces_per_token, h = piece % pieces_per_token;
+        bulk_load(ring + stage * slot_bytes + t * row_bytes + h * DIM * 2,
+                  k + (long long)(tok0 + key + t) * s.k_st + (long long)(head0 + h) * s.k_sh, piece_bytes, bar);
+      }
+    }
+    if (!ok && lane == 0 && device_status) atomicOr(device_status, FASTAV_DEV_WAIT_EXPIRED);
+    return;
+  }
+
+  // ---- consumers ---------------------------------------------------------------------------------------
   const int group = threadIdx.x / kLanes, lane = threadIdx.x % kLanes;
-  const int head = blockIdx.y * heads_per_block + group % heads_per_block;  // KV head of this lane group
+  const int head_local = group % heads_per_block, head = head0 + head_local;  // KV head of this lane group
   const int keys_per_step = kGroups / heads_per_block;
   const int key_lane = group / heads_per_block;
   const bool causal = (s.flags & FASTAV_CAUSAL) != 0;
   const int my_row = (lane >> kPlainBits) & (ROWS - 1);  // the row whose finished logit lands in this lane
   const bool writer = (lane & ((1 << kPlainBits) - 1)) == 0;
-  const uint16_t* kbase = k + (long long)tok0 * s.k_st + (long long)head * s.k_sh + lane * 8;
+  const uint32_t lane_off = head_local * DIM * 2 + lane * 16;
 
-  for (int pass0 = 0; pass0 < flat_rows; pass0 += ROWS) {
+  int it = 0;
+  for (int pass = 0; pass < passes; ++pass) {
+    const int pass0 = pass * ROWS;
     // Query rows of this pass: flat index f = r * G + (head within the group).
     float2 qv[ROWS][4];
 #pragma unroll
@@ -82,21 +140,22 @@ score_narrow_logits_kernel(Shapes s, const uint16_t* __restrict__ q, const int32
     const int limit = (causal && row_valid) ? q_idx[row0 + r_mine] : 0x7FFFFFFF;
     float* out = logits + ((long long)(head * s.group + (row_valid ? f_mine % s.group : 0)) * rq + r_mine) * s.total_tokens + tok0;
 
-    // The trip count is the same for every lane of the block (the shuffles below need whole warps).
-    for (int base = key_begin; base < key_end; base += keys_per_step * kUnroll) {
-      const int key0 = base + key_lane;
-      uint4 raw[kUnroll];
-#pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
-        const int key = key0 + u * keys_per_step;
-        raw[u] = make_uint4(0, 0, 0, 0);
-        if (key < key_end) raw[u] = __ldg(reinterpret_cast<const uint4*>(kbase + (long long)key * s.k_st));
-      }
-#pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
-        const int key = key0 + u * keys_per_step;
+    for (int sl = 0; sl < slots; ++sl, ++it) {
+      const int stage = it % kStages;
+      if (!ptx::mbar_wait_bounded(ptx::smem_u32(&full[stage]), (it / kStages) & 1, &abort_flag)) return;
+      const int key_base = key_begin + sl * kSlotKeys;
+      const uint32_t slot = ring + stage * slot_bytes + lane_off;
+      // The trip count is the same for every lane (the shuffles below need whole warps).
+#pragma unroll 2
+      for (int t0 = 0; t0 < kSlotKeys; t0 += keys_per_step) {
+        const int t = t0 + key_lane, key = key_base + t;
+        uint4 raw = make_uint4(0, 0, 0, 0);
+        if (t < kSlotKeys)
+          asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                       : "=r"(raw.x), "=r"(raw.y), "=r"(raw.z), "=r"(raw.w)
+                       : "r"(slot + t * row_bytes));
         float2 kv[4];
-        unpack8(raw[u], kv);
+        unpack8(raw, kv);
         float vals[ROWS];
 #pragma unroll
         for (int i = 0; i < ROWS; ++i) {
@@ -125,8 +184,11 @@ score_narrow_logits_kernel(Shapes s, const uint16_t* __restrict__ q, const int32
             vals[0] += __shfl_xor_sync(0xFFFFFFFFu, vals[0], off);
           }
         }
-        if (writer && row_valid && key < key_end) out[key] = key <= limit ? vals[0] * s.scale_log2 : -INFINITY;
+        // Tokens past the end of the chunk hold stale bytes of an earlier slot: computed, never written.
+        if (writer && row_valid && t < kSlotKeys && key < key_end) out[key] = key <= limit ? vals[0] * s.scale_log2 : -INFINITY;
       }
+      __syncwarp();
+      if ((threadIdx.x & 31) == 0) ptx::mbar_arrive(ptx::smem_u32(&empty[stage]));  // this warp is done with the slot
     }
   }
 }
@@ -226,22 +288,22 @@ __global__ void __launch_bounds__(kFinalizeThreads) score_narrow_finalize_kernel
 
 template <int DIM, int ROWS>
 cudaError_t launch_logits(const Shapes& s, const uint16_t* q, const int32_t* q_idx, const int32_t* cu_qlens, const uint16_t* k,
-                   const int32_t* cu_seqlens, float* logits, int rq, cudaStream_t stream) {
-  constexpr int kGroups = kThreads / (DIM / 8);
+                          const int32_t* cu_seqlens, float* logits, int rq, int32_t* device_status, cudaStream_t stream) {
+  constexpr int kGroups = kComputeThreads / (DIM / 8);
   // One block covers `hb` KV heads so that a step of the block reads whole contiguous token rows.
   int hb = 1;
   while (hb * 2 <= s.hkv && s.hkv % (hb * 2) == 0 && hb * 2 <= kGroups) hb *= 2;
-  const int keys_per_step = kGroups / hb;
-  const int quantum = keys_per_step * Unroll<ROWS>::value;
-  // Enough blocks to fill the machine a few times over, but never less than one unrolled step each.
-  const long long want_blocks = (long long)kNumSMs * 8;
-  long long chunk = ((long long)s.total_tokens * (s.hkv / hb) + want_blocks - 1) / want_blocks;
-  chunk = (chunk + quantum - 1) / quantum * quantum;
-  if (chunk < quantum) chunk = quantum;
-  if (chunk > 8 * quantum) chunk = 8 * quantum;
+  // Key chunk per block: a multiple of the slot size, about two blocks per SM over the whole batch, 64..1024 keys.
+  long long chunk = ((long long)s.total_tokens * (s.hkv / hb) + 2 * kNumSMs - 1) / (2 * kNumSMs);
+  chunk = (chunk + kSlotKeys - 1) / kSlotKeys * kSlotKeys;
+  if (chunk < 4 * kSlotKeys) chunk = 4 * kSlotKeys;
+  if (chunk > 64 * kSlotKeys) chunk = 64 * kSlotKeys;
+  const size_t smem = (size_t)kStages * kSlotKeys * hb * DIM * 2;
+  cudaError_t e = cudaFuncSetAttribute(score_narrow_logits_kernel<DIM, ROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
   const dim3 grid((unsigned)((s.max_seqlen + chunk - 1) / chunk), s.hkv / hb, s.batch);
-  return launch_chained(score_narrow_logits_kernel<DIM, ROWS>, grid, dim3(kThreads), 0, stream, s, q, q_idx, cu_qlens, k, cu_seqlens,
-                        logits, rq, hb, (int)chunk);
+  return launch_chained(score_narrow_logits_kernel<DIM, ROWS>, grid, dim3(kThreads), smem, stream, s, q, q_idx, cu_qlens, k, cu_seqlens,
+                        logits, rq, hb, (int)chunk, device_status);
 }
 
 }  // namespace
@@ -250,7 +312,7 @@ bool score_narrow_applies(const Shapes& s) { return s.max_qlen >= 1 && s.max_qle
 
 cudaError_t launch_score_narrow(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
                                 const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
-                                unsigned char* ws, cudaStream_t stream) {
+                                unsigned char* ws, int32_t* device_status, cudaStream_t stream) {
   const uint16_t* qq = static_cast<const uint16_t*>(q);
   const uint16_t* kk = static_cast<const uint16_t*>(k);
   float* logits = reinterpret_cast<float*>(ws + w.logits_off);
@@ -259,11 +321,11 @@ cudaError_t launch_score_narrow(const Shapes& s, const Workspace& w, const void*
   const bool four = s.max_qlen * s.group <= 4;
   cudaError_t e;
   if (s.dim == 128) {
-    e = four ? launch_logits<128, 4>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, stream)
-             : launch_logits<128, 8>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, stream);
+    e = four ? launch_logits<128, 4>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, device_status, stream)
+             : launch_logits<128, 8>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, device_status, stream);
   } else {
-    e = four ? launch_logits<64, 4>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, stream)
-             : launch_logits<64, 8>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, stream);
+    e = four ? launch_logits<64, 4>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, device_status, stream)
+             : launch_logits<64, 8>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, device_status, stream);
   }
   if (e != cudaSuccess) return e;
   if ((e = launch_chained(score_narrow_stats_kernel, dim3(s.hq * rq, s.batch), dim3(256), 0, stream, s, cu_qlens, cu_seqlens,
