@@ -61,6 +61,10 @@ cudaError_t launch_score_wide(const Shapes& s, const Workspace& w, const void* q
                               const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
                               unsigned char* ws, int32_t* device_status, cudaStream_t stream, bool* used);
 
+cudaError_t launch_logits_wide(const Shapes& s, const void* q, const int32_t* q_idx, const int32_t* cu_qlens, const void* k,
+                               const int32_t* cu_seqlens, float* logits, int rq, int32_t* device_status, cudaStream_t stream,
+                               bool* used);
+
 cudaError_t launch_select(const Shapes& s, const Workspace& w, const float* scores, const int32_t* cu_seqlens,
                           const int32_t* keep_counts, const uint8_t* protect, const int32_t* q_idx,
                           const int32_t* cu_qlens, int32_t* keep_idx, int32_t* cu_keep, unsigned char* ws,

@@ -320,7 +320,16 @@ cudaError_t launch_score_narrow(const Shapes& s, const Workspace& w, const void*
   const int rq = s.max_qlen;
   const bool four = s.max_qlen * s.group <= 4;
   cudaError_t e;
-  if (s.dim == 128) {
+  // The logits come from a skinny tensor-core MMA over TMA-streamed K tiles where that kernel takes the shapes
+  // (and the caller did not ask for the CUDA-core kernel); otherwise from the lane-group kernel above.
+  bool by_mma = false;
+  if ((s.flags & FASTAV_SCORE_PATH_MASK) != FASTAV_SCORE_PATH_NARROW && score_wide_applies(s)) {
+    e = launch_logits_wide(s, q, q_idx, cu_qlens, k, cu_seqlens, logits, rq, device_status, stream, &by_mma);
+    if (e != cudaSuccess) return e;
+  }
+  if (by_mma) {
+    e = cudaSuccess;
+  } else if (s.dim == 128) {
     e = four ? launch_logits<128, 4>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, device_status, stream)
              : launch_logits<128, 8>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, device_status, stream);
   } else {
@@ -336,7 +345,7 @@ cudaError_t launch_score_narrow(const Shapes& s, const Workspace& w, const void*
                           s.hq * rq * sizeof(float), stream, s, cu_qlens, cu_seqlens, (const float*)logits, rq, (const float*)lse,
                           scores_out)) != cudaSuccess)
     return e;
-  count_launches(3);
+  count_launches(by_mma ? 2 : 3);
   return cudaGetLastError();
 }
 

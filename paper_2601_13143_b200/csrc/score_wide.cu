@@ -228,7 +228,7 @@ score_wide_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
                   const int32_t* __restrict__ q_idx, const int32_t* __restrict__ cu_qlens,
                   const int32_t* __restrict__ cu_seqlens, int chunk_tiles, int stat_chunks, int rc_max, int rows_per_chunk,
                   float2* __restrict__ stats, const float* __restrict__ lse, float* __restrict__ partial,
-                  int32_t* device_status) {
+                  float* __restrict__ logits, int rq, int32_t* device_status) {
   using L = Layout<DIM>;
   extern __shared__ unsigned char smem_raw[];
   pdl_trigger();
@@ -349,7 +349,7 @@ score_wide_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
   if (warp == 0) {
     // ---- TMA producer: one elected lane streams query tiles and K tiles ---------------------------
     if (lane == 0) {
-      if constexpr (SWEEP == 1) pdl_wait();  // q and k may be what the previous kernel in the stream wrote
+      if constexpr (SWEEP != 2) pdl_wait();  // first kernel of a chain: q and k may be what the previous kernel in the stream wrote
       int tile_no = 0, q_gen = 0;  // K tiles / query tiles issued so far
       bool ok = true;
       for (int u = 0; u < n_units && ok; ++u) {
@@ -505,6 +505,52 @@ score_wide_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
         if (ok && row_valid) {
           const long long rh = (long long)(un.row0 + r) * s.hq + un.g * s.group + f % s.group;
           stats[rh * stat_chunks + un.kc * 2 + h] = make_float2(zmax * s.scale_log2, sum2.x + sum2.y);
+        }
+      }
+    } else if constexpr (SWEEP == 0) {
+      // Logits only (few scored rows: the matrix-vector case done as a skinny MMA, bound by streaming K).
+      // Thread <-> key, warpgroup w owns the query-row columns [32 w, 32 w + 32) and writes their scaled,
+      // masked logits to the [Hq, rq, N] workspace; consecutive lanes write consecutive tokens.
+      int tile_no = 0;
+      bool ok = true;
+      int* slot_of = reinterpret_cast<int*>(ctl.neg_lse[warp - 2]);  // per column: head * rq + scored row
+      int* limit = ctl.limit[warp - 2];
+      for (int u = 0; u < n_units && ok; ++u) {
+        const Unit un = ctl.units[u];
+        const int key_begin = un.kc * chunk_keys;
+        const int tiles = (min(un.n - key_begin, chunk_keys) + kTileKeys - 1) / kTileKeys;
+        const int my_cols = max(0, min(32, un.rows_here - wg * 32));
+        if (un.new_q) {
+          __syncwarp();
+          const int f = un.rc * rows_per_chunk + wg * 32 + lane;
+          const int r = f / s.group;
+          slot_of[lane] = (un.g * s.group + f % s.group) * rq + r;
+          limit[lane] = (causal && lane < my_cols) ? q_idx[un.row0 + r] : INT_MAX;
+          __syncwarp();
+        }
+        float* out = logits + un.tok0;
+        for (int t = 0; t < tiles; ++t, ++tile_no) {
+          const int i = tile_no & 1;
+          ok = ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.tmem_full[i]), (tile_no >> 1) & 1, abort);
+          if (!ok) break;
+          ptx::tc_fence_after_sync();
+          const int key = key_begin + t * kTileKeys + my_lane;
+          if (my_cols > 0) {
+            uint32_t v[32];
+            ptx::tmem_ld32(lane_addr + i * 256 + wg * 32, v);
+            tmem_ld_wait_for(v);
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive(ptx::smem_u32(&ctl.tmem_empty[i]));
+            if (key < un.n) {
+#pragma unroll
+              for (int c = 0; c < 32; ++c)
+                if (c < my_cols)
+                  out[(long long)slot_of[c] * s.total_tokens + key] = key <= limit[c] ? __uint_as_float(v[c]) * s.scale_log2 : -INFINITY;
+            }
+          } else {
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive(ptx::smem_u32(&ctl.tmem_empty[i]));
+          }
         }
       }
     } else {
@@ -683,6 +729,35 @@ bool make_map(const void* ptr, int dim, int heads, long long rows, long long st,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Persistent grid and key chunk: one block per SM; chunks sized so that a block gets about a dozen units (fine
+// enough to balance, and never more than its table holds).
+void plan_units(const Shapes& s, int rc_max, int* grid_out, int* chunk_tiles_out) {
+  const long long tiles_upper = (long long)s.total_tokens / kTileKeys + s.batch;  // >= sum over sequences of ceil(n / 128)
+  const long long tile_units = tiles_upper * s.hkv * rc_max;
+  const int grid = (int)(tile_units < kNumSMs ? tile_units : kNumSMs);
+  long long chunk_tiles = (tile_units + (long long)grid * 14 - 1) / ((long long)grid * 14);
+  if (chunk_tiles < 1) chunk_tiles = 1;
+  // units <= hkv * rc_max * (tokens / chunk + batch); keep the per-block share within the table
+  while (((long long)s.hkv * rc_max * (s.total_tokens / (chunk_tiles * kTileKeys) + s.batch) + grid - 1) / grid + 1 > kMaxUnits)
+    ++chunk_tiles;
+  *grid_out = grid;
+  *chunk_tiles_out = (int)chunk_tiles;
+}
+
+template <int DIM>
+cudaError_t run_logits(const Shapes& s, const CUtensorMap& k_map, const CUtensorMap& q_map, const int32_t* q_idx,
+                       const int32_t* cu_qlens, const int32_t* cu_seqlens, float* logits, int rq, int32_t* device_status,
+                       cudaStream_t stream) {
+  int grid, chunk_tiles;
+  plan_units(s, 1, &grid, &chunk_tiles);
+  const int smem = Layout<DIM>::kTotal;
+  cudaError_t e = cudaFuncSetAttribute(score_wide_kernel<DIM, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  return launch_chained(score_wide_kernel<DIM, 0>, dim3(grid), dim3(kThreads), smem, stream, k_map, q_map, s, q_idx, cu_qlens,
+                        cu_seqlens, chunk_tiles, 0, 1, wide_rows_per_chunk(s.group), (float2*)nullptr, (const float*)nullptr,
+                        (float*)nullptr, logits, rq, device_status);
+}
+
 template <int DIM>
 cudaError_t run(const Shapes& s, const Workspace& w, const CUtensorMap& k_map, const CUtensorMap& q_map, const int32_t* q_idx,
                 const int32_t* cu_qlens, const int32_t* cu_seqlens, float* scores_out, unsigned char* ws,
@@ -692,33 +767,25 @@ cudaError_t run(const Shapes& s, const Workspace& w, const CUtensorMap& k_map, c
   float* partial = reinterpret_cast<float*>(ws + w.partial_off);
   const int rows_per_chunk = wide_rows_per_chunk(s.group);
   const int rc_max = wide_row_chunks(s.max_qlen, s.group);
-  // One persistent block per SM.  Key chunks are sized so that a block gets about a dozen units (fine
-  // enough to balance, and never more than its table holds).
-  const long long tiles_upper = (long long)s.total_tokens / kTileKeys + s.batch;  // >= sum over sequences of ceil(n / 128)
-  const long long tile_units = tiles_upper * s.hkv * rc_max;
-  const int grid = (int)(tile_units < kNumSMs ? tile_units : kNumSMs);
-  long long chunk_tiles = (tile_units + (long long)grid * 14 - 1) / ((long long)grid * 14);
-  if (chunk_tiles < 1) chunk_tiles = 1;
-  // units <= hkv * rc_max * (tokens / chunk + batch); keep the per-block share within the table
-  while (((long long)s.hkv * rc_max * (s.total_tokens / (chunk_tiles * kTileKeys) + s.batch) + grid - 1) / grid + 1 > kMaxUnits)
-    ++chunk_tiles;
-  const int chunk_keys = (int)chunk_tiles * kTileKeys;
+  int grid, chunk_tiles;
+  plan_units(s, rc_max, &grid, &chunk_tiles);
+  const int chunk_keys = chunk_tiles * kTileKeys;
   const int stat_chunks = 2 * ((s.max_seqlen + chunk_keys - 1) / chunk_keys);  // (max, sum) entries per (row, head)
   const int smem = Layout<DIM>::kTotal;
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(score_wide_kernel<DIM, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(score_wide_kernel<DIM, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) return e;
   if ((e = launch_chained(score_wide_kernel<DIM, 1>, dim3(grid), dim3(kThreads), smem, stream, k_map, q_map, s, q_idx, cu_qlens,
-                          cu_seqlens, (int)chunk_tiles, stat_chunks, rc_max, rows_per_chunk, stats, (const float*)nullptr,
-                          (float*)nullptr, device_status)) != cudaSuccess)
+                          cu_seqlens, chunk_tiles, stat_chunks, rc_max, rows_per_chunk, stats, (const float*)nullptr,
+                          (float*)nullptr, (float*)nullptr, 0, device_status)) != cudaSuccess)
     return e;
   const int warps = s.total_q * s.hq;
   if ((e = launch_chained(score_wide_merge_kernel, dim3((warps + 7) / 8), dim3(256), 0, stream, s, cu_qlens, cu_seqlens,
                           (const float2*)stats, stat_chunks, chunk_keys, lse)) != cudaSuccess)
     return e;
   if ((e = launch_chained(score_wide_kernel<DIM, 2>, dim3(grid), dim3(kThreads), smem, stream, k_map, q_map, s, q_idx, cu_qlens,
-                          cu_seqlens, (int)chunk_tiles, stat_chunks, rc_max, rows_per_chunk, (float2*)nullptr, (const float*)lse,
-                          partial, device_status)) != cudaSuccess)
+                          cu_seqlens, chunk_tiles, stat_chunks, rc_max, rows_per_chunk, (float2*)nullptr, (const float*)lse,
+                          partial, (float*)nullptr, 0, device_status)) != cudaSuccess)
     return e;
   if ((e = launch_chained(score_wide_finalize_kernel, dim3((s.max_seqlen + kFinalizeThreads - 1) / kFinalizeThreads, s.batch),
                           dim3(kFinalizeThreads), 0, stream, s,
@@ -744,6 +811,19 @@ bool score_wide_applies(const Shapes& s) {
   const auto ok_stride = [](long long v) { return v > 0 && v % 8 == 0 && (v >> 36) == 0; };
   return s.max_qlen >= 1 && s.total_q >= 1 && s.max_seqlen >= 1 && (s.dim == 64 || s.dim == 128) && s.group <= 32 &&
          ok_stride(s.k_st) && ok_stride(s.k_sh) && ok_stride(s.q_st) && ok_stride(s.q_sh);
+}
+
+// Logits [Hq, rq, N] of a batch with at most rq <= 4 scored rows per sequence, by the tensor-core kernel.
+cudaError_t launch_logits_wide(const Shapes& s, const void* q, const int32_t* q_idx, const int32_t* cu_qlens, const void* k,
+                               const int32_t* cu_seqlens, float* logits, int rq, int32_t* device_status, cudaStream_t stream,
+                               bool* used) {
+  CUtensorMap k_map, q_map;
+  *used = rq * s.group <= 128 && make_map(k, s.dim, s.hkv, s.total_tokens, s.k_st, s.k_sh, 1, kTileKeys, &k_map) &&
+          make_map(q, s.dim, s.hq, s.total_q, s.q_st, s.q_sh, s.group, 8, &q_map);
+  if (!*used) return cudaSuccess;
+  count_launches(1);
+  if (s.dim == 128) return run_logits<128>(s, k_map, q_map, q_idx, cu_qlens, cu_seqlens, logits, rq, device_status, stream);
+  return run_logits<64>(s, k_map, q_map, q_idx, cu_qlens, cu_seqlens, logits, rq, device_status, stream);
 }
 
 cudaError_t launch_score_wide(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
