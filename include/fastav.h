@@ -121,7 +121,13 @@ int32_t fastav_workspace_bytes(const fastav_params* params, size_t* out_bytes);
  *   cu_qlens   [B+1] int32
  *   k          [N, Hkv, head_dim] bf16
  *   cu_seqlens [B+1] int32
- *   lse_opt    reserved, pass NULL
+ *   lse_opt    [total_q, Hq] fp32 or NULL.  Optional log-sum-exp of each scored row and head, as the
+ *              layer's own attention kernel returns it for these rows: natural logarithm of
+ *              sum_{j' in V(r)} exp(scale <q, k_j'>), same scale and mask as here (-inf for a row that sees
+ *              no key).  The method does not rely on the attention map (Section 1: it stays compatible
+ *              with FlashAttention-style kernels), and those kernels produce exactly this by-product;
+ *              with it the scores need one sweep over K instead of two.  The result is the same
+ *              quantity (a wrong lse gives wrong scores; nothing checks it).
  *   scores_out [N] fp32 (written for every token; a sequence with R_b = 0 gets zeros)
  */
 int32_t fastav_score(const fastav_params* params, const void* q, const int32_t* q_idx, const int32_t* cu_qlens,

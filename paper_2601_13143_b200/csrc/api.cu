@@ -161,19 +161,19 @@ bool score_path_ok(const Shapes& s) {
 // Shape-based choice: few scored rows -> matrix-vector path; otherwise the tensor-core path; the
 // CUDA-core tiles take whatever is left (and whatever the TMA descriptor cannot express).
 cudaError_t launch_score(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
-                         const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
-                         unsigned char* ws, int32_t* device_status, cudaStream_t stream) {
+                         const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, const float* lse_in,
+                         float* scores_out, unsigned char* ws, int32_t* device_status, cudaStream_t stream) {
   const unsigned forced = s.flags & FASTAV_SCORE_PATH_MASK;
-  if (forced == FASTAV_SCORE_PATH_GENERIC) return launch_score_generic(s, w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out, ws, stream);
+  if (forced == FASTAV_SCORE_PATH_GENERIC) return launch_score_generic(s, w, q, q_idx, cu_qlens, k, cu_seqlens, lse_in, scores_out, ws, stream);
   if (score_narrow_applies(s) && (forced == 0 || forced == FASTAV_SCORE_PATH_NARROW))
-    return launch_score_narrow(s, w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out, ws, device_status, stream);
+    return launch_score_narrow(s, w, q, q_idx, cu_qlens, k, cu_seqlens, lse_in, scores_out, ws, device_status, stream);
   if (score_wide_applies(s)) {
     bool used = false;
-    const cudaError_t e = launch_score_wide(s, w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out, ws, device_status, stream, &used);
+    const cudaError_t e = launch_score_wide(s, w, q, q_idx, cu_qlens, k, cu_seqlens, lse_in, scores_out, ws, device_status, stream, &used);
     if (used || e != cudaSuccess) return e;
     if (forced == FASTAV_SCORE_PATH_WIDE) return cudaErrorNotSupported;
   }
-  return launch_score_generic(s, w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out, ws, stream);
+  return launch_score_generic(s, w, q, q_idx, cu_qlens, k, cu_seqlens, lse_in, scores_out, ws, stream);
 }
 
 }  // namespace fastav
@@ -213,13 +213,12 @@ int32_t fastav_score(const fastav_params* params, const void* q, const int32_t* 
                      void* workspace, size_t workspace_bytes, int32_t* device_status, void* stream) {
   int32_t rc = check_params(params);
   if (rc != FASTAV_OK) return rc;
-  if (lse_opt) return FASTAV_ERR_UNSUPPORTED;
   if ((rc = check_score_args(params, q, q_idx, cu_qlens, k, cu_seqlens, scores_out)) != FASTAV_OK) return rc;
   const Workspace w = plan_workspace(*params);
   if ((rc = check_workspace(w, workspace, workspace_bytes)) != FASTAV_OK) return rc;
   if (!score_path_ok(make_shapes(*params))) return FASTAV_ERR_UNSUPPORTED;
   if (params->total_tokens == 0) return FASTAV_OK;
-  const cudaError_t e = launch_score(make_shapes(*params), w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out,
+  const cudaError_t e = launch_score(make_shapes(*params), w, q, q_idx, cu_qlens, k, cu_seqlens, lse_opt, scores_out,
                                      static_cast<unsigned char*>(workspace), device_status, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? FASTAV_OK : cuda_failed(e);
 }
@@ -273,7 +272,7 @@ int32_t fastav_prune(const fastav_params* params, const void* q, const int32_t* 
   unsigned char* ws = static_cast<unsigned char*>(workspace);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e = cudaSuccess;
-  if (params->total_tokens > 0) e = launch_score(s, w, q, q_idx, cu_qlens, k, cu_seqlens, scores_out, ws, device_status, st);
+  if (params->total_tokens > 0) e = launch_score(s, w, q, q_idx, cu_qlens, k, cu_seqlens, nullptr, scores_out, ws, device_status, st);
   if (e == cudaSuccess)
     e = launch_select(s, w, scores_out, cu_seqlens, keep_counts, protect_opt, q_idx, cu_qlens, keep_idx_out, cu_keep_out, ws,
                       device_status, st);

@@ -38,19 +38,25 @@ Workspace plan_workspace(const fastav_params& p);
 
 // ---- launchers (each returns cudaGetLastError() after its launches) -------------------------
 cudaError_t launch_score(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
-                         const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
-                         unsigned char* ws, int32_t* device_status, cudaStream_t stream);
+                         const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, const float* lse_in,
+                         float* scores_out, unsigned char* ws, int32_t* device_status, cudaStream_t stream);
 
+// `lse_in` (optional, everywhere below): the caller's natural-log log-sum-exp per (scored row, head); when
+// given, the softmax statistics are not recomputed.
 cudaError_t launch_score_generic(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
-                                 const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
-                                 unsigned char* ws, cudaStream_t stream);
+                                 const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, const float* lse_in,
+                                 float* scores_out, unsigned char* ws, cudaStream_t stream);
+
+// lse_ws[i] = log2(e) * lse_in[i] (the kernels work in base-2 units); a non-finite entry (a row that saw no
+// key) becomes +inf, i.e. the row contributes nothing.
+cudaError_t launch_lse_import(const Shapes& s, const float* lse_in, float* lse_ws, cudaStream_t stream);
 
 // Few scored rows per sequence (the paper's fine stage scores the last token only): matrix-vector path.
 constexpr int kNarrowMaxRows = 4;
 bool score_narrow_applies(const Shapes& s);
 cudaError_t launch_score_narrow(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
-                                const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
-                                unsigned char* ws, int32_t* device_status, cudaStream_t stream);
+                                const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, const float* lse_in,
+                                float* scores_out, unsigned char* ws, int32_t* device_status, cudaStream_t stream);
 
 // Many scored rows per sequence: tensor-core path (tcgen05 + TMA).  `*used` is false when the TMA
 // descriptor for K could not be built; nothing was launched then and the caller takes another path.
@@ -58,8 +64,8 @@ int wide_rows_per_chunk(int group);
 int wide_row_chunks(int max_qlen, int group);
 bool score_wide_applies(const Shapes& s);
 cudaError_t launch_score_wide(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
-                              const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
-                              unsigned char* ws, int32_t* device_status, cudaStream_t stream, bool* used);
+                              const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, const float* lse_in,
+                              float* scores_out, unsigned char* ws, int32_t* device_status, cudaStream_t stream, bool* used);
 
 cudaError_t launch_logits_wide(const Shapes& s, const void* q, const int32_t* q_idx, const int32_t* cu_qlens, const void* k,
                                const int32_t* cu_seqlens, float* logits, int rq, int32_t* device_status, cudaStream_t stream,

@@ -237,9 +237,19 @@ __global__ void __launch_bounds__(256) score_finalize_kernel(Shapes s, const int
   }
 }
 
+__global__ void __launch_bounds__(256) lse_import_kernel(int count, const float* __restrict__ lse_in, float* __restrict__ lse_ws) {
+  pdl_trigger();
+  pdl_wait();
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  const float v = lse_in[i];
+  lse_ws[i] = (v == v && fabsf(v) != INFINITY) ? v * kLog2e : INFINITY;
+}
+
 template <int DIM>
 cudaError_t run(const Shapes& s, const Workspace& w, const uint16_t* q, const int32_t* q_idx, const int32_t* cu_qlens,
-                const uint16_t* k, const int32_t* cu_seqlens, float* scores_out, unsigned char* ws, cudaStream_t stream) {
+                const uint16_t* k, const int32_t* cu_seqlens, const float* lse_in, float* scores_out, unsigned char* ws,
+                cudaStream_t stream) {
   float2* stats = reinterpret_cast<float2*>(ws + w.stats_off);
   float* lse = reinterpret_cast<float*>(ws + w.lse_off);
   float* partial = reinterpret_cast<float*>(ws + w.partial_off);
@@ -249,11 +259,16 @@ cudaError_t run(const Shapes& s, const Workspace& w, const uint16_t* q, const in
   if ((e = cudaFuncSetAttribute(score_tile_accumulate_kernel<DIM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
   if (s.total_q > 0 && s.max_seqlen > 0) {
     const dim3 grid(w.stat_tiles, s.hkv, s.batch);
-    score_tile_stats_kernel<DIM><<<grid, kThreads, smem, stream>>>(s, q, q_idx, cu_qlens, k, cu_seqlens, stats, w.stat_tiles);
-    const int warps = s.total_q * s.hq;
-    score_merge_stats_kernel<<<(warps + 7) / 8, 256, 0, stream>>>(s, cu_qlens, cu_seqlens, stats, w.stat_tiles, lse);
+    if (lse_in) {
+      if ((e = launch_lse_import(s, lse_in, lse, stream)) != cudaSuccess) return e;
+    } else {
+      score_tile_stats_kernel<DIM><<<grid, kThreads, smem, stream>>>(s, q, q_idx, cu_qlens, k, cu_seqlens, stats, w.stat_tiles);
+      const int warps = s.total_q * s.hq;
+      score_merge_stats_kernel<<<(warps + 7) / 8, 256, 0, stream>>>(s, cu_qlens, cu_seqlens, stats, w.stat_tiles, lse);
+      count_launches(2);
+    }
     score_tile_accumulate_kernel<DIM><<<grid, kThreads, smem, stream>>>(s, q, q_idx, cu_qlens, k, cu_seqlens, lse, partial);
-    count_launches(3);
+    count_launches(1);
   }
   if (s.max_seqlen > 0) {
     const dim3 grid((s.max_seqlen + 255) / 256, s.batch);
@@ -265,13 +280,20 @@ cudaError_t run(const Shapes& s, const Workspace& w, const uint16_t* q, const in
 
 }  // namespace
 
+cudaError_t launch_lse_import(const Shapes& s, const float* lse_in, float* lse_ws, cudaStream_t stream) {
+  const int count = s.total_q * s.hq;
+  if (count <= 0) return cudaSuccess;
+  count_launches(1);
+  return launch_chained(lse_import_kernel, dim3((count + 255) / 256), dim3(256), 0, stream, count, lse_in, lse_ws);
+}
+
 cudaError_t launch_score_generic(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
-                                 const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
-                                 unsigned char* ws, cudaStream_t stream) {
+                                 const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, const float* lse_in,
+                                 float* scores_out, unsigned char* ws, cudaStream_t stream) {
   const uint16_t* qq = static_cast<const uint16_t*>(q);
   const uint16_t* kk = static_cast<const uint16_t*>(k);
-  if (s.dim == 128) return run<128>(s, w, qq, q_idx, cu_qlens, kk, cu_seqlens, scores_out, ws, stream);
-  return run<64>(s, w, qq, q_idx, cu_qlens, kk, cu_seqlens, scores_out, ws, stream);
+  if (s.dim == 128) return run<128>(s, w, qq, q_idx, cu_qlens, kk, cu_seqlens, lse_in, scores_out, ws, stream);
+  return run<64>(s, w, qq, q_idx, cu_qlens, kk, cu_seqlens, lse_in, scores_out, ws, stream);
 }
 
 }  // namespace fastav

@@ -311,8 +311,8 @@ cudaError_t launch_logits(const Shapes& s, const uint16_t* q, const int32_t* q_i
 bool score_narrow_applies(const Shapes& s) { return s.max_qlen >= 1 && s.max_qlen <= kNarrowMaxRows && s.hq <= 256; }
 
 cudaError_t launch_score_narrow(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
-                                const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
-                                unsigned char* ws, int32_t* device_status, cudaStream_t stream) {
+                                const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, const float* lse_in,
+                                float* scores_out, unsigned char* ws, int32_t* device_status, cudaStream_t stream) {
   const uint16_t* qq = static_cast<const uint16_t*>(q);
   const uint16_t* kk = static_cast<const uint16_t*>(k);
   float* logits = reinterpret_cast<float*>(ws + w.logits_off);
@@ -337,15 +337,16 @@ cudaError_t launch_score_narrow(const Shapes& s, const Workspace& w, const void*
              : launch_logits<64, 8>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, device_status, stream);
   }
   if (e != cudaSuccess) return e;
-  if ((e = launch_chained(score_narrow_stats_kernel, dim3(s.hq * rq, s.batch), dim3(256), 0, stream, s, cu_qlens, cu_seqlens,
-                          (const float*)logits, rq, lse)) != cudaSuccess)
-    return e;
+  if (lse_in) e = launch_lse_import(s, lse_in, lse, stream);
+  else e = launch_chained(score_narrow_stats_kernel, dim3(s.hq * rq, s.batch), dim3(256), 0, stream, s, cu_qlens, cu_seqlens,
+                          (const float*)logits, rq, lse);
+  if (e != cudaSuccess) return e;
   if ((e = launch_chained(score_narrow_finalize_kernel, dim3((s.max_seqlen + kFinalizeThreads - 1) / kFinalizeThreads, s.batch),
                           dim3(kFinalizeThreads),
                           s.hq * rq * sizeof(float), stream, s, cu_qlens, cu_seqlens, (const float*)logits, rq, (const float*)lse,
                           scores_out)) != cudaSuccess)
     return e;
-  count_launches(by_mma ? 2 : 3);
+  count_launches((by_mma ? 0 : 1) + (lse_in ? 0 : 1) + 1);  // the tensor-core logits and the lse import count themselves
   return cudaGetLastError();
 }
 

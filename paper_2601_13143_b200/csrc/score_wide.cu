@@ -760,7 +760,7 @@ cudaError_t run_logits(const Shapes& s, const CUtensorMap& k_map, const CUtensor
 
 template <int DIM>
 cudaError_t run(const Shapes& s, const Workspace& w, const CUtensorMap& k_map, const CUtensorMap& q_map, const int32_t* q_idx,
-                const int32_t* cu_qlens, const int32_t* cu_seqlens, float* scores_out, unsigned char* ws,
+                const int32_t* cu_qlens, const int32_t* cu_seqlens, const float* lse_in, float* scores_out, unsigned char* ws,
                 int32_t* device_status, cudaStream_t stream) {
   float2* stats = reinterpret_cast<float2*>(ws + w.stats_off);
   float* lse = reinterpret_cast<float*>(ws + w.lse_off);
@@ -775,14 +775,20 @@ cudaError_t run(const Shapes& s, const Workspace& w, const CUtensorMap& k_map, c
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(score_wide_kernel<DIM, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(score_wide_kernel<DIM, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) return e;
-  if ((e = launch_chained(score_wide_kernel<DIM, 1>, dim3(grid), dim3(kThreads), smem, stream, k_map, q_map, s, q_idx, cu_qlens,
-                          cu_seqlens, chunk_tiles, stat_chunks, rc_max, rows_per_chunk, stats, (const float*)nullptr,
-                          (float*)nullptr, (float*)nullptr, 0, device_status)) != cudaSuccess)
-    return e;
-  const int warps = s.total_q * s.hq;
-  if ((e = launch_chained(score_wide_merge_kernel, dim3((warps + 7) / 8), dim3(256), 0, stream, s, cu_qlens, cu_seqlens,
-                          (const float2*)stats, stat_chunks, chunk_keys, lse)) != cudaSuccess)
-    return e;
+  if (lse_in) {
+    // The caller already has log-sum-exp per (row, head) (the layer's attention kernel returns it): one sweep.
+    if ((e = launch_lse_import(s, lse_in, lse, stream)) != cudaSuccess) return e;
+  } else {
+    if ((e = launch_chained(score_wide_kernel<DIM, 1>, dim3(grid), dim3(kThreads), smem, stream, k_map, q_map, s, q_idx, cu_qlens,
+                            cu_seqlens, chunk_tiles, stat_chunks, rc_max, rows_per_chunk, stats, (const float*)nullptr,
+                            (float*)nullptr, (float*)nullptr, 0, device_status)) != cudaSuccess)
+      return e;
+    const int warps = s.total_q * s.hq;
+    if ((e = launch_chained(score_wide_merge_kernel, dim3((warps + 7) / 8), dim3(256), 0, stream, s, cu_qlens, cu_seqlens,
+                            (const float2*)stats, stat_chunks, chunk_keys, lse)) != cudaSuccess)
+      return e;
+    count_launches(2);
+  }
   if ((e = launch_chained(score_wide_kernel<DIM, 2>, dim3(grid), dim3(kThreads), smem, stream, k_map, q_map, s, q_idx, cu_qlens,
                           cu_seqlens, chunk_tiles, stat_chunks, rc_max, rows_per_chunk, (float2*)nullptr, (const float*)lse,
                           partial, (float*)nullptr, 0, device_status)) != cudaSuccess)
@@ -791,7 +797,7 @@ cudaError_t run(const Shapes& s, const Workspace& w, const CUtensorMap& k_map, c
                           dim3(kFinalizeThreads), 0, stream, s,
                           cu_seqlens, cu_qlens, rc_max, rows_per_chunk, (const float*)partial, scores_out)) != cudaSuccess)
     return e;
-  count_launches(4);
+  count_launches(2);
   return cudaGetLastError();
 }
 
@@ -827,14 +833,14 @@ cudaError_t launch_logits_wide(const Shapes& s, const void* q, const int32_t* q_
 }
 
 cudaError_t launch_score_wide(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
-                              const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, float* scores_out,
-                              unsigned char* ws, int32_t* device_status, cudaStream_t stream, bool* used) {
+                              const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, const float* lse_in,
+                              float* scores_out, unsigned char* ws, int32_t* device_status, cudaStream_t stream, bool* used) {
   CUtensorMap k_map, q_map;
   *used = make_map(k, s.dim, s.hkv, s.total_tokens, s.k_st, s.k_sh, 1, kTileKeys, &k_map) &&
           make_map(q, s.dim, s.hq, s.total_q, s.q_st, s.q_sh, s.group, 8, &q_map);
   if (!*used) return cudaSuccess;  // the caller falls back to the CUDA-core path
-  if (s.dim == 128) return run<128>(s, w, k_map, q_map, q_idx, cu_qlens, cu_seqlens, scores_out, ws, device_status, stream);
-  return run<64>(s, w, k_map, q_map, q_idx, cu_qlens, cu_seqlens, scores_out, ws, device_status, stream);
+  if (s.dim == 128) return run<128>(s, w, k_map, q_map, q_idx, cu_qlens, cu_seqlens, lse_in, scores_out, ws, device_status, stream);
+  return run<64>(s, w, k_map, q_map, q_idx, cu_qlens, cu_seqlens, lse_in, scores_out, ws, device_status, stream);
 }
 
 }  // namespace fastav

@@ -80,8 +80,6 @@ def test_null_and_workspace_errors_enqueue_nothing(lib):
     assert rc == fastav.FASTAV_ERR_WORKSPACE              # not 256-byte aligned
     rc = lib.fastav_score(ctypes.byref(p), ctypes.c_void_p(0x1008), fake, fake, fake, fake, null, fake, fake, ctypes.c_size_t(1 << 30), null, null)
     assert rc == fastav.FASTAV_ERR_UNSUPPORTED            # q not 16-byte aligned
-    rc = lib.fastav_score(ctypes.byref(p), fake, fake, fake, fake, fake, fake, fake, fake, ctypes.c_size_t(1 << 30), null, null)
-    assert rc == fastav.FASTAV_ERR_UNSUPPORTED            # lse_opt is reserved
     p_bad = _params()
     p_bad.k_stride_head = 60                               # shorter than a row
     rc = lib.fastav_score(ctypes.byref(p_bad), fake, fake, fake, fake, fake, null, fake, fake, ctypes.c_size_t(1 << 30), null, null)

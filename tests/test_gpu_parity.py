@@ -80,6 +80,43 @@ def test_score_matches_oracle(lens, rows, hq, hkv, d, causal, path):
     assert torch.equal(first.view(torch.int32), buf.scores.view(torch.int32))
 
 
+def _natural_lse(p):
+    """log sum_j exp(scale q.k_j) over the keys each scored row may see, per (row, head), in float64 on the CPU
+    (what an attention kernel would hand back for these rows)."""
+    cu, cuq = p.cu_seqlens.tolist(), p.cu_qlens.tolist()
+    hq, hkv = p.q.shape[1], p.k.shape[1]
+    out = torch.full((p.q.shape[0], hq), float("-inf"), dtype=torch.float64)
+    for b in range(len(cu) - 1):
+        k = p.k[cu[b]:cu[b + 1]].double().repeat_interleave(hq // hkv, dim=1)            # [n, Hq, d]
+        for r in range(cuq[b], cuq[b + 1]):
+            z = torch.einsum("hd,nhd->hn", p.q[r].double(), k) * p.softmax_scale          # [Hq, n]
+            if p.causal:
+                z = z[:, :int(p.q_idx[r]) + 1]
+            if z.shape[1]:
+                out[r] = torch.logsumexp(z, dim=1)
+    return out.float()
+
+
+@pytest.mark.parametrize("lens,rows,hq,hkv,d", [([300, 40], [3, 1], 8, 2, 64), ([1000], [64], 8, 2, 128), ([777, 130], [40, 9], 28, 4, 128)])
+@pytest.mark.parametrize("path", ["auto", "generic"])
+def test_score_with_caller_provided_lse(lens, rows, hq, hkv, d, path):
+    """The attention kernel's log-sum-exp replaces the first sweep; the scores are the same quantity."""
+    p = W.random_problem(seed=11, lens=lens, rows=rows, keeps=[n // 2 for n in lens], num_q_heads=hq, num_kv_heads=hkv,
+                         head_dim=d, hidden=64)
+    buf = parity.to_device(p, extra_flags=SCORE_PATHS[path])
+    lse = _natural_lse(p).cuda()
+    launches = fastav.fastav_kernel_launches()
+    fastav.fastav_score(buf.params, buf.q, buf.q_idx, buf.cu_qlens, buf.k, buf.cu_seqlens, buf.scores, buf.workspace,
+                        buf.device_status, lse_opt=lse)
+    with_lse = fastav.fastav_kernel_launches() - launches
+    torch.cuda.synchronize()
+    parity.assert_scores_close(buf.scores, parity.oracle_scores(p), f"lse given, {path}")
+    launches = fastav.fastav_kernel_launches()
+    buf.score()
+    torch.cuda.synchronize()
+    assert with_lse <= fastav.fastav_kernel_launches() - launches       # never more work than the self-contained path
+
+
 def test_score_softmax_scale_one_is_eq4_as_printed():
     p = W.random_problem(seed=3, lens=[50], rows=[1], keeps=[25], num_q_heads=4, num_kv_heads=2, head_dim=64, hidden=64)
     p.softmax_scale = 1.0
