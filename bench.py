@@ -34,6 +34,7 @@ if ROOT not in sys.path:
 
 from paper_2601_13143_b200 import workloads as W  # noqa: E402
 from paper_2601_13143_b200 import flops as F  # noqa: E402
+from paper_2601_13143_b200 import replicas as R  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
@@ -312,12 +313,9 @@ def main():
     launches = fastav.fastav_kernel_launches() - launches0
     step_ms = [a.elapsed_time(b) for a, b in zip(starts, stops)]
     total_ms = sum(step_ms)
-    if dist is not None:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = R.max_over_ranks(total_ms, dist, device)
     ms_per_step = total_ms / args.steps
-    value = world * tokens_per_step / (ms_per_step * 1e-3)
+    value = R.aggregate_throughput(tokens_per_step, ms_per_step, world)
 
     # ---- per-kernel times of the same steps (separate entry points, events in between) ----
     phase_ms = [{"score": 0.0, "select": 0.0, "compact": 0.0} for _ in stages]
@@ -392,11 +390,8 @@ def main():
         torch.cuda.synchronize()
         barrier()
         e2e_ms = a.elapsed_time(b) / e2e_steps
-        if dist is not None:
-            t = torch.tensor([e2e_ms], dtype=torch.float64, device=device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
-        e2e = {"value": world * tokens_per_step / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms, "steps": e2e_steps,
+        e2e_ms = R.max_over_ranks(e2e_ms, dist, device)
+        e2e = {"value": R.aggregate_throughput(tokens_per_step, e2e_ms, world), "unit": "tokens/s", "ms_per_step": e2e_ms, "steps": e2e_steps,
                "h2d_bytes_per_step": sum(h["h2d"] for h in chain), "d2h_bytes_per_step": sum(h["d2h"] for h in chain),
                "api": "fastav_prune_host (pinned host buffers)"}
         del chain
