@@ -154,6 +154,25 @@ int32_t fastav_select(const fastav_params* params, const float* scores, const in
                       size_t workspace_bytes, int32_t* device_status, void* stream);
 
 /*
+ * Keep set given by rule instead of by score.  The paper's deployed GLOBAL stage (Section 2.2, "Global
+ * pruning"; Section 3.1, implementation details) is positional: the rollout analysis fixes once which
+ * positions matter (e.g. the first 10 audio tokens, the first 4 frames) and at the middle layer every
+ * other audio/video token is dropped without looking at scores.  The caller states such a rule as a mask;
+ * this call turns it into the keep list that fastav_compact consumes:
+ *
+ *   keep_mask    [N] uint8            token j of the packed batch survives iff keep_mask[j] != 0
+ *   keep_idx_out [total_keep] int32   survivors, ascending per sequence (same convention as fastav_select)
+ *   cu_keep_out  [B+1] int32          prefix sums of the per-sequence survivor counts
+ *
+ * params.total_keep is the capacity of keep_idx_out: survivors beyond it are not written, cu_keep_out is
+ * clamped to it and FASTAV_DEV_K_CLAMPED is set.  Of params only batch, total_tokens, total_keep and flags
+ * are read.  Workspace: 256-byte aligned, at least 4 * batch bytes (rounded up to 256).
+ */
+int32_t fastav_select_mask(const fastav_params* params, const uint8_t* keep_mask, const int32_t* cu_seqlens,
+                           int32_t* keep_idx_out, int32_t* cu_keep_out, void* workspace, size_t workspace_bytes,
+                           int32_t* device_status, void* stream);
+
+/*
  * Survivor layout (what "iteratively refining the token set" in Section 2.2 leaves for the next
  * layer): output row cu_keep[b] + i is input row cu_seqlens[b] + keep_idx[cu_keep[b] + i] of
  *

@@ -121,6 +121,19 @@ def select(scores, cu_seqlens, keep_counts, protect_mask=None, protect_rows=Fals
     return keep_idx[:total], cu_keep
 
 
+def select_mask(keep_mask, cu_seqlens, global_index=False):
+    """Keep list of a rule-given mask (Section 2.2, "Global pruning": the deployed global stage keeps
+    fixed positions): the kept tokens of each sequence in ascending order.  Returns (keep_idx, cu_keep)."""
+    keep_mask = np.asarray(keep_mask)
+    cu_seqlens = _i32(cu_seqlens)
+    parts, cu_keep = [], [0]
+    for b in range(len(cu_seqlens) - 1):
+        kept = [j for j in range(int(cu_seqlens[b + 1] - cu_seqlens[b])) if keep_mask[cu_seqlens[b] + j] != 0]
+        parts.append(np.asarray(kept, dtype=np.int32) + (int(cu_seqlens[b]) if global_index else 0))
+        cu_keep.append(cu_keep[-1] + len(kept))
+    return (np.concatenate(parts) if parts else np.zeros(0, dtype=np.int32)).astype(np.int32), np.asarray(cu_keep, dtype=np.int32)
+
+
 def compact(keep_idx, cu_keep, cu_seqlens, hidden=None, pos=None, k=None, v=None, global_index=False):
     """Gather the survivors' rows.  Returns dict(hidden, pos, k, v) of packed outputs (None where
     the input was None)."""

@@ -259,6 +259,103 @@ cudaError_t launch_select(const Shapes& s, const Workspace& w, const float* scor
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
+// ---- keep set given as a mask (the paper's positional global rule) ---------------------------------
+namespace {
+
+// counts[b] = number of kept tokens of sequence b.
+__global__ void __launch_bounds__(256) mask_count_kernel(int batch, const uint8_t* __restrict__ keep_mask,
+                                                         const int32_t* __restrict__ cu_seqlens, int32_t* __restrict__ counts) {
+  __shared__ int warp_sums[8];
+  pdl_trigger();
+  pdl_wait();
+  pdl_acquire(keep_mask);
+  const int b = blockIdx.x;
+  const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
+  int c = 0;
+  for (int j = threadIdx.x; j < n; j += 256) c += keep_mask[tok0 + j] != 0;
+  c = __reduce_add_sync(0xFFFFFFFFu, c);
+  if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = c;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int total = 0;
+    for (int w = 0; w < 8; ++w) total += warp_sums[w];
+    counts[b] = total;
+  }
+}
+
+// Survivors of sequence b in ascending order, after those of the sequences before it.
+__global__ void __launch_bounds__(kThreads) mask_emit_kernel(Shapes s, const uint8_t* __restrict__ keep_mask,
+                                                             const int32_t* __restrict__ cu_seqlens,
+                                                             const int32_t* __restrict__ counts, int32_t* __restrict__ keep_idx,
+                                                             int32_t* __restrict__ cu_keep, int32_t* device_status) {
+  __shared__ unsigned warp_a[kWarps];
+  __shared__ int base_sh;
+  pdl_trigger();
+  pdl_wait();
+  pdl_acquire(counts);
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
+  if (tid == 0) base_sh = 0;
+  __syncthreads();
+  int part = 0;
+  for (int i = tid; i < b; i += kThreads) part += counts[i];
+  if (part) atomicAdd(&base_sh, part);
+  __syncthreads();
+  const int base = base_sh;
+  if (tid == 0) {
+    cu_keep[b + 1] = min(base + counts[b], s.total_keep);
+    if (b == 0) cu_keep[0] = 0;
+    if (base + counts[b] > s.total_keep && device_status) atomicOr(device_status, FASTAV_DEV_K_CLAMPED);
+  }
+  const bool global_idx = (s.flags & FASTAV_KEEP_IDX_GLOBAL) != 0;
+  const int per = (n + kThreads - 1) / kThreads;
+  const int j0 = min(n, tid * per), j1 = min(n, j0 + per);
+  unsigned mine = 0;
+  for (int j = j0; j < j1; ++j) mine += keep_mask[tok0 + j] != 0;
+  unsigned incl = mine;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const unsigned t = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+    if (lane >= d) incl += t;
+  }
+  if (lane == 31) warp_a[warp] = incl;
+  __syncthreads();
+  unsigned before = incl - mine;
+  for (int w = 0; w < warp; ++w) before += warp_a[w];
+  for (int j = j0; j < j1; ++j)
+    if (keep_mask[tok0 + j]) {
+      const int out = base + (int)before++;
+      if (out < s.total_keep) keep_idx[out] = global_idx ? tok0 + j : j;  // never past the caller's buffer
+    }
+}
+
+}  // namespace
+}  // namespace fastav
+
+extern "C" int32_t fastav_select_mask(const fastav_params* p, const uint8_t* keep_mask, const int32_t* cu_seqlens,
+                                      int32_t* keep_idx_out, int32_t* cu_keep_out, void* workspace, size_t workspace_bytes,
+                                      int32_t* device_status, void* stream) {
+  using namespace fastav;
+  if (!p || p->batch < 1 || p->total_tokens < 0 || p->total_keep < 0 || p->total_keep > p->total_tokens) return FASTAV_ERR_INVALID_ARG;
+  if (!cu_seqlens || !cu_keep_out || (p->total_tokens > 0 && !keep_mask) || (p->total_keep > 0 && !keep_idx_out))
+    return FASTAV_ERR_INVALID_ARG;
+  const size_t need = align_up((size_t)p->batch * sizeof(int32_t), 256);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < need) return FASTAV_ERR_WORKSPACE;
+  Shapes s{};
+  s.batch = p->batch; s.total_tokens = p->total_tokens; s.max_seqlen = p->max_seqlen; s.total_keep = p->total_keep;
+  s.flags = p->flags;
+  int32_t* counts = static_cast<int32_t*>(workspace);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e = launch_chained(mask_count_kernel, dim3(s.batch), dim3(256), 0, st, s.batch, keep_mask, cu_seqlens, counts);
+  if (e == cudaSuccess)
+    e = launch_chained(mask_emit_kernel, dim3(s.batch), dim3(kThreads), 0, st, s, keep_mask, cu_seqlens, (const int32_t*)counts,
+                       keep_idx_out, cu_keep_out, device_status);
+  count_launches(2);
+  return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? FASTAV_OK : FASTAV_ERR_CUDA;
+}
+
+namespace fastav {
+
 // ---- fastav_select_noalloc: the same selection with its scratch inside the library ----------
 //
 // The radix select keeps one 32-bit key per token.  fastav_select puts them in shared memory or in

@@ -36,7 +36,7 @@ FASTAV_ERR_TIMEOUT = -5
 
 EXPORTS = ("fastav_version", "fastav_status_string", "fastav_last_cuda_error", "fastav_workspace_bytes",
            "fastav_score", "fastav_select", "fastav_compact", "fastav_prune", "fastav_host_arena_bytes",
-           "fastav_prune_host", "fastav_kernel_launches", "fastav_select_noalloc")
+           "fastav_prune_host", "fastav_kernel_launches", "fastav_select_noalloc", "fastav_select_mask")
 
 
 class fastav_params(ctypes.Structure):
@@ -106,6 +106,8 @@ def library() -> ctypes.CDLL:
         lib.fastav_prune_host.argtypes = [pp, vp, i32p, i32p, vp, vp, i32p, i32p, vp, vp, i32p, vp, i32p, i32p, vp, i32p,
                                           vp, vp, i32p, vp, ctypes.c_size_t, vp]
         lib.fastav_kernel_launches.restype = ctypes.c_int64
+        lib.fastav_select_mask.restype = ctypes.c_int32
+        lib.fastav_select_mask.argtypes = [pp, vp, i32p, i32p, i32p, vp, ctypes.c_size_t, i32p, vp]
         lib.fastav_select_noalloc.restype = ctypes.c_int32
         lib.fastav_select_noalloc.argtypes = [pp, vp, i32p, i32p, vp, i32p, i32p, i32p, i32p, i32p, vp]
         _lib = lib
@@ -185,6 +187,13 @@ def fastav_select(params, scores, cu_seqlens, keep_counts, protect_opt, q_idx, c
     _check(library().fastav_select(ctypes.byref(params), _p(scores), _p(cu_seqlens), _p(keep_counts), _p(protect_opt),
                                    _p(q_idx), _p(cu_qlens), _p(keep_idx_out), _p(cu_keep_out), ws, ws_bytes,
                                    _p(device_status), _stream(stream)), "fastav_select")
+
+
+def fastav_select_mask(params, keep_mask, cu_seqlens, keep_idx_out, cu_keep_out, workspace, device_status=None, stream=None) -> None:
+    """Keep list of a rule-given keep mask (the paper's positional global stage)."""
+    ws, ws_bytes = _ws(workspace)
+    _check(library().fastav_select_mask(ctypes.byref(params), _p(keep_mask), _p(cu_seqlens), _p(keep_idx_out), _p(cu_keep_out),
+                                        ws, ws_bytes, _p(device_status), _stream(stream)), "fastav_select_mask")
 
 
 NOALLOC_MAX_TOKENS = 1 << 20

@@ -275,3 +275,17 @@ def random_problem(seed: int, lens: list[int], rows: list[int], keeps: list[int]
     return PruneInputs(model=model, q=q, k=k, v=v, hidden=h, pos=pos, cu_seqlens=cu, cu_qlens=cu_q, q_idx=q_idx,
                        keep_counts=torch.tensor(keeps, dtype=torch.int32), softmax_scale=1.0 / math.sqrt(head_dim),
                        causal=True, protect_rows=False)
+
+
+def positional_keep_mask(modality: torch.Tensor, cu_seqlens: torch.Tensor, keep_first: dict[int, int]) -> torch.Tensor:
+    """Keep mask of a positional rule of the kind the paper deploys at its global stage: of every modality
+    named in ``keep_first`` only the first m tokens of each sequence survive (e.g. ``{MOD_AUDIO: 10}`` keeps
+    the first 10 audio tokens); tokens of all other modalities survive.  Input construction only."""
+    mask = torch.ones_like(modality, dtype=torch.uint8)
+    cu = cu_seqlens.tolist()
+    for b in range(len(cu) - 1):
+        seg = modality[cu[b]:cu[b + 1]]
+        for mod, m in keep_first.items():
+            idx = torch.nonzero(seg == mod).flatten()
+            mask[cu[b] + idx[m:]] = 0
+    return mask

@@ -226,6 +226,58 @@ def test_select_sequence_longer_than_shared_memory():
     assert _select_case([n, 100], [n // 3, 50], scores=np.concatenate([scores, rng.random(100).astype(np.float32)])) == 0
 
 
+def test_positional_global_prune_keeps_first_audio_tokens():
+    """The paper's deployed global stage: a positional rule (here: only the first 10 audio tokens survive,
+    everything else is kept) -> keep list -> survivor layout, against the oracle."""
+    w = W.WORKLOADS["c2_global_2k"]
+    p = W.make_stage(w, 0)
+    mask = W.positional_keep_mask(p.modality, p.cu_seqlens, {W.MOD_AUDIO: 10})
+    ref_idx, ref_cu = oracle.select_mask(mask.numpy(), p.cu_seqlens.numpy())
+    kept = int(ref_cu[-1])
+    assert kept == p.total_tokens - (256 - 10)
+    ref = oracle.compact(ref_idx, ref_cu, p.cu_seqlens.numpy(), bf16_bits(p.hidden), p.pos.numpy(), bf16_bits(p.k), bf16_bits(p.v))
+    p.keep_counts = torch.tensor([kept], dtype=torch.int32)
+    buf = parity.to_device(p, flags=0)
+    buf.keep_idx.fill_(-7)
+    fastav.fastav_select_mask(buf.params, mask.cuda(), buf.cu_seqlens, buf.keep_idx, buf.cu_keep, buf.workspace, buf.device_status)
+    buf.compact()
+    assert _sync_status(buf) == 0
+    assert buf.cu_keep.cpu().tolist() == ref_cu.tolist()
+    assert buf.keep_idx.cpu().numpy()[:kept].tolist() == ref_idx.tolist()
+    for name in ("hidden", "pos", "k", "v"):
+        parity.assert_bits_equal(getattr(buf, name + "_out"), ref[name], name)
+
+
+def test_select_mask_ragged_global_indices_and_capacity_clamp():
+    rng = np.random.default_rng(9)
+    lens = [5, 0, 2000, 1, 333]
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    mask = (rng.random(cu[-1]) < 0.5).astype(np.uint8)
+    for glob in (False, True):
+        ref_idx, ref_cu = oracle.select_mask(mask, cu, global_index=glob)
+        total = int(ref_cu[-1])
+        params = fastav.make_params(batch=len(lens), total_tokens=int(cu[-1]), max_seqlen=max(lens), total_q=0, max_qlen=0,
+                                    total_keep=total, max_keep=total, num_q_heads=4, num_kv_heads=2, head_dim=64, hidden=64,
+                                    flags=fastav.FASTAV_KEEP_IDX_GLOBAL if glob else 0)
+        keep_idx = torch.full((total + 8,), -7, dtype=torch.int32, device="cuda")
+        cu_keep = torch.full((len(lens) + 1,), -7, dtype=torch.int32, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+        fastav.fastav_select_mask(params, torch.as_tensor(mask).cuda(), torch.as_tensor(cu).cuda(), keep_idx, cu_keep, ws, status)
+        torch.cuda.synchronize()
+        assert cu_keep.cpu().tolist() == ref_cu.tolist() and int(status) == 0
+        got = keep_idx.cpu().numpy()
+        assert got[:total].tolist() == ref_idx.tolist() and (got[total:] == -7).all()
+    # a keep buffer that is too small: nothing written past it, the clamp is reported
+    params.total_keep = params.max_keep = total - 50
+    keep_idx.fill_(-7)
+    status.zero_()
+    fastav.fastav_select_mask(params, torch.as_tensor(mask).cuda(), torch.as_tensor(cu).cuda(), keep_idx, cu_keep, ws, status)
+    torch.cuda.synchronize()
+    assert int(status) & fastav.FASTAV_DEV_K_CLAMPED and int(cu_keep[-1]) == total - 50
+    assert (keep_idx.cpu().numpy()[total - 50:] == -7).all()
+
+
 # ---- compact ----------------------------------------------------------------------------------
 
 @pytest.mark.parametrize("hkv,d,hid", [(2, 64, 64), (4, 128, 3584), (8, 128, 4096), (1, 64, 8)])

@@ -291,3 +291,21 @@ def test_flops_column_of_table_4(golden_dir):
     seen = oflops.token_schedule(1000, 6, {3: 500, 4: 400})
     assert seen == [1000, 1000, 1000, 500, 400, 400]
     assert oflops.removed_count(1024, 0.2) == 204 and oflops.removed_count(820, 0.2) == 164
+
+
+def test_mask_selection_equals_score_selection_on_indicator_scores():
+    """A keep mask is the special case of the score rule in which kept tokens score 1, dropped ones 0 and
+    k is the number of ones: the two oracle routes must agree (ties among the ones go to the lower index,
+    which is ascending order)."""
+    rng = np.random.default_rng(3)
+    lens = [0, 1, 17, 64, 5]
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    mask = (rng.random(cu[-1]) < 0.4).astype(np.uint8)
+    mask[cu[2]:cu[2] + 3] = 1
+    counts = [int(mask[cu[b]:cu[b + 1]].sum()) for b in range(len(lens))]
+    by_mask, cu_mask = oracle.select_mask(mask, cu)
+    by_score, cu_score = oracle.select(mask.astype(np.float32), cu, counts)
+    assert cu_mask.tolist() == cu_score.tolist() == np.concatenate([[0], np.cumsum(counts)]).tolist()
+    assert by_mask.tolist() == by_score.tolist()
+    glob, _ = oracle.select_mask(mask, cu, global_index=True)
+    assert glob.tolist() == np.nonzero(mask)[0].tolist()
