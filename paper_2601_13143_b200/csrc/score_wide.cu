@@ -38,7 +38,7 @@ constexpr int kGroups = 4;        // softmax warpgroups: four warps per schedule
 constexpr int kThreads = 64 + 128 * kGroups;  // warp 0: TMA, warp 1: MMA, warps 2-17: softmax
 constexpr int kTmemCols = 512;
 constexpr int kMaxUnits = 48;       // work units one block may be given (the host sizes key chunks accordingly)
-constexpr int kCtrlBytes = 16 * 1024;
+constexpr int kCtrlBytes = 18 * 1024;
 
 template <int DIM>
 struct Layout {
@@ -192,6 +192,7 @@ struct Control {
   int n_units;
   int start_b, start_off;
   int warp_sums[kThreads / 32];
+  int seq_first_unit[kThreads + 1];            // batch <= kThreads: first unit of every sequence, then the total
   alignas(16) float neg_lse[4 * kGroups][64];  // sweep 2, per softmax warp: -lse of its query-row columns (-inf: padding)
   alignas(16) int limit[4 * kGroups][64];      // sweep 2, per softmax warp: last key each column's row may see
   float sums[2][kGroups - 1][kTileKeys];       // sweep 2: per accumulator, the partial sums of warpgroups 1-3
@@ -244,11 +245,34 @@ score_wide_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
 
   // ---- this block's share of the work: units [u0, u1) of the list ordered by (sequence, KV head,
   //      row chunk, key chunk), so that consecutive units mostly share their query tile -------------
-  int total_units = 0;
-  for (int b0 = 0; b0 < s.batch; b0 += kThreads) {
-    const int b = b0 + threadIdx.x;
-    total_units += block_sum(b < s.batch ? units_of_sequence(s, cu_seqlens, cu_qlens, b, rows_per_chunk, chunk_keys) : 0,
-                             ctl.warp_sums);
+  const bool table = s.batch <= kThreads;  // one sequence per thread: the unit table can be built in parallel
+  int total_units = 0, my_units = 0, my_excl = 0;
+  if (table) {
+    const int b = threadIdx.x;
+    my_units = b < s.batch ? units_of_sequence(s, cu_seqlens, cu_qlens, b, rows_per_chunk, chunk_keys) : 0;
+    int incl = my_units;  // inclusive scan inside the warp, then across warps through shared memory
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int t = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+      if (lane >= d) incl += t;
+    }
+    if (lane == 31) ctl.warp_sums[warp] = incl;
+    __syncthreads();
+    int warp_base = 0;
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) {
+      if (w < warp) warp_base += ctl.warp_sums[w];
+      total_units += ctl.warp_sums[w];
+    }
+    my_excl = warp_base + incl - my_units;
+    ctl.seq_first_unit[b] = my_excl;  // first unit of sequence b in the global order
+    if (b == 0) ctl.seq_first_unit[kThreads] = total_units;
+  } else {
+    for (int b0 = 0; b0 < s.batch; b0 += kThreads) {
+      const int b = b0 + threadIdx.x;
+      total_units += block_sum(b < s.batch ? units_of_sequence(s, cu_seqlens, cu_qlens, b, rows_per_chunk, chunk_keys) : 0,
+                               ctl.warp_sums);
+    }
   }
   const int u0 = (int)((long long)total_units * blockIdx.x / gridDim.x);
   const int u1 = (int)((long long)total_units * (blockIdx.x + 1) / gridDim.x);
@@ -256,12 +280,47 @@ score_wide_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
     pdl_wait();
     return;
   }
-  {
+  const int n_mine = min(u1 - u0, kMaxUnits);
+  // Unit `target` of the global order -> what to work on.  `b` is its sequence, `off` its index inside it.
+  auto describe = [&](int b, int off, Unit& un) {
+    un.tok0 = cu_seqlens[b];
+    un.n = cu_seqlens[b + 1] - un.tok0;
+    un.row0 = cu_qlens[b];
+    const int flat_rows = (cu_qlens[b + 1] - un.row0) * s.group;
+    const int row_chunks = (flat_rows + rows_per_chunk - 1) / rows_per_chunk;
+    const int key_chunks = (un.n + chunk_keys - 1) / chunk_keys;
+    const int grc = off / key_chunks;
+    un.g = grc / row_chunks;
+    un.rc = grc % row_chunks;
+    un.kc = off % key_chunks;
+    un.rows_here = min(rows_per_chunk, flat_rows - un.rc * rows_per_chunk);
+    un.new_q = 1;
+  };
+  if (table) {
+    __syncthreads();
+    if (threadIdx.x < n_mine) {
+      const int target = u0 + threadIdx.x;
+      int lo = 0, hi = s.batch;  // smallest hi with first_unit[hi] > target; the sequence is hi - 1 (empty ones are skipped)
+      while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        const int first_next = mid + 1 < s.batch ? ctl.seq_first_unit[mid + 1] : total_units;
+        if (first_next > target) hi = mid; else lo = mid + 1;
+      }
+      Unit un;
+      describe(lo, target - ctl.seq_first_unit[lo], un);
+      ctl.units[threadIdx.x] = un;
+    }
+    __syncthreads();
+    if (threadIdx.x > 0 && threadIdx.x < n_mine) {  // same sequence, KV head and row chunk as the unit before: same query tile
+      const Unit &a = ctl.units[threadIdx.x - 1], &c = ctl.units[threadIdx.x];
+      if (a.tok0 == c.tok0 && a.g == c.g && a.rc == c.rc) ctl.units[threadIdx.x].new_q = 0;
+    }
+  } else {
     int before = 0;  // units of the sequences before the current batch slice
     for (int b0 = 0; b0 < s.batch; b0 += kThreads) {
       const int b = b0 + threadIdx.x;
       const int mine = b < s.batch ? units_of_sequence(s, cu_seqlens, cu_qlens, b, rows_per_chunk, chunk_keys) : 0;
-      int incl = mine;  // inclusive scan inside the warp, then across warps through shared memory
+      int incl = mine;
 #pragma unroll
       for (int d = 1; d < 32; d <<= 1) {
         const int t = __shfl_up_sync(0xFFFFFFFFu, incl, d);
@@ -283,37 +342,24 @@ score_wide_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
       }
       before += slice_total;
     }
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    // Walk the units of this block and write them down for every role.
-    int b = ctl.start_b, off = ctl.start_off, count = 0, prev_b = -1, prev_grc = -1;
-    int tok0 = 0, n = 0, row0 = 0, flat_rows = 0, row_chunks = 0, key_chunks = 0, loaded_b = -1;
-    for (int u = u0; u < u1 && count < kMaxUnits; ++u) {
-      for (;;) {
-        if (b != loaded_b) {  // the (slow, dependent) global loads happen once per sequence
-          tok0 = cu_seqlens[b];
-          n = cu_seqlens[b + 1] - tok0;
-          row0 = cu_qlens[b];
-          flat_rows = (cu_qlens[b + 1] - row0) * s.group;
-          row_chunks = (flat_rows + rows_per_chunk - 1) / rows_per_chunk;
-          key_chunks = (n + chunk_keys - 1) / chunk_keys;
-          loaded_b = b;
+    __syncthreads();
+    if (threadIdx.x == 0) {  // very large batches: one thread walks this block's units
+      int b = ctl.start_b, off = ctl.start_off;
+      for (int i = 0; i < n_mine; ++i) {
+        while (off >= units_of_sequence(s, cu_seqlens, cu_qlens, b, rows_per_chunk, chunk_keys)) {
+          ++b;  // sequence exhausted (or empty): on to the next one
+          off = 0;
         }
-        if (n > 0 && flat_rows > 0 && off < s.hkv * row_chunks * key_chunks) break;
-        ++b;  // sequence exhausted (or empty): on to the next one
-        off = 0;
+        Unit un;
+        describe(b, off, un);
+        if (i > 0 && ctl.units[i - 1].tok0 == un.tok0 && ctl.units[i - 1].g == un.g && ctl.units[i - 1].rc == un.rc) un.new_q = 0;
+        ctl.units[i] = un;
+        ++off;
       }
-      const int grc = off / key_chunks;
-      Unit un;
-      un.tok0 = tok0; un.n = n; un.row0 = row0;
-      un.g = grc / row_chunks; un.rc = grc % row_chunks; un.kc = off % key_chunks;
-      un.rows_here = min(rows_per_chunk, flat_rows - un.rc * rows_per_chunk);
-      un.new_q = (b != prev_b || grc != prev_grc) ? 1 : 0;
-      prev_b = b; prev_grc = grc;
-      ctl.units[count++] = un;
-      ++off;
     }
+  }
+  if (threadIdx.x == 0) {
+    const int count = n_mine;
     ctl.n_units = count;
     for (int i = 0; i < kStages; ++i) {
       ptx::mbar_init(ptx::smem_u32(&ctl.full_k[i]), 1);
