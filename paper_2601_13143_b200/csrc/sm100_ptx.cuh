@@ -48,10 +48,13 @@ constexpr uint64_t kWaitLimitNs = 500ull * 1000 * 1000;
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
-  for (uint32_t spin = 1;; ++spin) {
-    if (mbar_try_wait(bar, parity)) return true;
+  for (;;) {
+    // a short tight run of attempts (each may suspend the thread for a while in hardware), then the checks
+#pragma unroll 1
+    for (int i = 0; i < 16; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
     if (*abort) return false;
-    if ((spin & 63u) == 0 && global_timer_ns() - t0 > kWaitLimitNs) {
+    if (global_timer_ns() - t0 > kWaitLimitNs) {
       *abort = 1;
       return false;
     }
