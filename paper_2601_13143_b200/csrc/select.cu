@@ -85,15 +85,15 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
   pdl_acquire(scores);
 
   // Keys.
-  for (int j0 = tid; j0 < n; j0 += kThreads * 8) {
-    float v[8];  // eight independent loads in flight per thread: one block serves a whole sequence
+  for (int j0 = tid; j0 < n; j0 += kThreads * 16) {
+    float v[16];  // sixteen independent loads in flight per thread: one block serves a whole sequence
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
+    for (int u = 0; u < 16; ++u) {
       const int j = j0 + u * kThreads;
       v[u] = j < n ? __ldg(scores + tok0 + j) : 0.f;
     }
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
+    for (int u = 0; u < 16; ++u) {
       const int j = j0 + u * kThreads;
       if (j < n) {
         unsigned key = order_key(v[u]);
@@ -186,8 +186,15 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
       }
       if (lane == 0) sh.warp_a[warp] = incl;
       __syncthreads();
-      unsigned above_warp = 0;
-      for (int w = warp + 1; w < kWarps; ++w) above_warp += sh.warp_a[w];
+      // keys in the bins of higher warps: suffix sum of the 32 warp totals with shuffles (every warp does the same)
+      unsigned suffix = sh.warp_a[lane];
+      const unsigned own_total = suffix;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const unsigned t = __shfl_down_sync(0xFFFFFFFFu, suffix, d);
+        if (lane + d < 32) suffix += t;
+      }
+      const unsigned above_warp = __shfl_sync(0xFFFFFFFFu, suffix - own_total, warp);
       const unsigned above_me = above_warp + incl - (h0 + h1);  // keys in bins above this thread's two
       const unsigned rem = (unsigned)sh.remaining;
       __syncthreads();  // everyone has read `remaining` before the one owner rewrites it
@@ -223,7 +230,17 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
   if (lane == 31) { sh.warp_a[warp] = gt_incl; sh.warp_b[warp] = eq_incl; }
   __syncthreads();
   unsigned gt_before = gt_incl - my_gt, eq_before = eq_incl - my_eq;
-  for (int w = 0; w < warp; ++w) { gt_before += sh.warp_a[w]; eq_before += sh.warp_b[w]; }
+  {  // plus the totals of the warps before this one: prefix sums of the 32 warp totals with shuffles
+    unsigned pa = sh.warp_a[lane], pb = sh.warp_b[lane];
+    const unsigned ta = pa, tb = pb;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const unsigned a = __shfl_up_sync(0xFFFFFFFFu, pa, d), c = __shfl_up_sync(0xFFFFFFFFu, pb, d);
+      if (lane >= d) { pa += a; pb += c; }
+    }
+    gt_before += __shfl_sync(0xFFFFFFFFu, pa - ta, warp);
+    eq_before += __shfl_sync(0xFFFFFFFFu, pb - tb, warp);
+  }
   for (int j = j0; j < j1; ++j) {
     const unsigned key = keys[slot<kKeysInShared>(j)];
     const bool gt = key > T, eq = key == T;
