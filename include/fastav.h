@@ -52,6 +52,8 @@ extern "C" {
 #define FASTAV_CAUSAL 1u              /* scored row r sees keys j <= q_idx[r] only (the model's own mask) */
 #define FASTAV_PROTECT_QUERY_ROWS 2u  /* the scored rows' tokens always survive (and count toward k_b) */
 #define FASTAV_KEEP_IDX_GLOBAL 4u     /* keep_idx holds indices into the packed batch, not sequence-local ones */
+#define FASTAV_SELECT_LOWEST 0x800u   /* fastav_select keeps the k_b LOWEST-scoring tokens instead: the "prune the most attended
+                                         tokens" control of the paper's ablations (Tables 2 and 3, "Top attentive") */
 
 /* Diagnostics: force one implementation of fastav_score instead of the shape-based choice.  A forced
  * path that does not support the shapes makes the call fail with FASTAV_ERR_UNSUPPORTED. */
@@ -247,6 +249,15 @@ int32_t fastav_select_noalloc(const fastav_params* params, const float* scores, 
                               const int32_t* keep_counts, const uint8_t* protect_opt, const int32_t* q_idx,
                               const int32_t* cu_qlens, int32_t* keep_idx_out, int32_t* cu_keep_out,
                               int32_t* device_status, void* stream);
+
+/*
+ * Diagnostic (the paper has no counterpart): enqueues a one-block kernel that waits, with the same bounded
+ * wait the scoring and compaction kernels use, on a barrier nothing ever completes.  After limit_ms
+ * (1..1000) milliseconds the wait gives up, the kernel sets FASTAV_DEV_WAIT_EXPIRED in *device_status and
+ * exits normally; the CUDA context stays usable.  It shows what a stuck copy or MMA would turn into: an error
+ * bit, not a hang.
+ */
+int32_t fastav_selftest_bounded_wait(int32_t limit_ms, int32_t* device_status, void* stream);
 
 /*
  * Number of kernels this library has launched in this process so far (a diagnostic counter; the

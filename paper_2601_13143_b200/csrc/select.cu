@@ -84,7 +84,8 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
   pdl_wait();  // the scores are the previous kernel's output
   pdl_acquire(scores);
 
-  // Keys.
+  // Keys.  Under FASTAV_SELECT_LOWEST the ranking is reversed by negating the scores (ties still go to the lower index).
+  const bool lowest = (s.flags & FASTAV_SELECT_LOWEST) != 0;
   for (int j0 = tid; j0 < n; j0 += kThreads * 16) {
     float v[16];  // sixteen independent loads in flight per thread: one block serves a whole sequence
 #pragma unroll
@@ -96,7 +97,7 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
     for (int u = 0; u < 16; ++u) {
       const int j = j0 + u * kThreads;
       if (j < n) {
-        unsigned key = order_key(v[u]);
+        unsigned key = order_key(lowest ? -v[u] : v[u]);
         if (key == kProtectedKey) key = kProtectedKey - 1;  // only a NaN pattern lands here
         if (protect && protect[tok0 + j]) key = kProtectedKey;
         keys[slot<kKeysInShared>(j)] = key;

@@ -16,6 +16,7 @@ from . import build as _build
 FASTAV_CAUSAL = 1
 FASTAV_PROTECT_QUERY_ROWS = 2
 FASTAV_KEEP_IDX_GLOBAL = 4
+FASTAV_SELECT_LOWEST = 0x800
 
 FASTAV_SCORE_PATH_GENERIC = 0x100
 FASTAV_SCORE_PATH_NARROW = 0x200
@@ -36,7 +37,7 @@ FASTAV_ERR_TIMEOUT = -5
 
 EXPORTS = ("fastav_version", "fastav_status_string", "fastav_last_cuda_error", "fastav_workspace_bytes",
            "fastav_score", "fastav_select", "fastav_compact", "fastav_prune", "fastav_host_arena_bytes",
-           "fastav_prune_host", "fastav_kernel_launches", "fastav_select_noalloc", "fastav_select_mask")
+           "fastav_prune_host", "fastav_kernel_launches", "fastav_select_noalloc", "fastav_select_mask", "fastav_selftest_bounded_wait")
 
 
 class fastav_params(ctypes.Structure):
@@ -108,6 +109,8 @@ def library() -> ctypes.CDLL:
         lib.fastav_kernel_launches.restype = ctypes.c_int64
         lib.fastav_select_mask.restype = ctypes.c_int32
         lib.fastav_select_mask.argtypes = [pp, vp, i32p, i32p, i32p, vp, ctypes.c_size_t, i32p, vp]
+        lib.fastav_selftest_bounded_wait.restype = ctypes.c_int32
+        lib.fastav_selftest_bounded_wait.argtypes = [ctypes.c_int32, i32p, vp]
         lib.fastav_select_noalloc.restype = ctypes.c_int32
         lib.fastav_select_noalloc.argtypes = [pp, vp, i32p, i32p, vp, i32p, i32p, i32p, i32p, i32p, vp]
         _lib = lib
@@ -194,6 +197,11 @@ def fastav_select_mask(params, keep_mask, cu_seqlens, keep_idx_out, cu_keep_out,
     ws, ws_bytes = _ws(workspace)
     _check(library().fastav_select_mask(ctypes.byref(params), _p(keep_mask), _p(cu_seqlens), _p(keep_idx_out), _p(cu_keep_out),
                                         ws, ws_bytes, _p(device_status), _stream(stream)), "fastav_select_mask")
+
+
+def fastav_selftest_bounded_wait(limit_ms: int, device_status, stream=None) -> None:
+    """Enqueue the bounded-wait self-test (a wait that cannot succeed; it must end with the error bit set)."""
+    _check(library().fastav_selftest_bounded_wait(int(limit_ms), _p(device_status), _stream(stream)), "fastav_selftest_bounded_wait")
 
 
 NOALLOC_MAX_TOKENS = 1 << 20

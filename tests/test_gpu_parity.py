@@ -154,13 +154,14 @@ def test_score_strided_qkv_views():
 
 # ---- select -----------------------------------------------------------------------------------
 
-def _select_case(lens, keeps, scores, protect=None, rows=None, q_idx=None, global_idx=False, protect_rows=False):
+def _select_case(lens, keeps, scores, protect=None, rows=None, q_idx=None, global_idx=False, protect_rows=False, lowest=False):
     cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
     rows = [0] * len(lens) if rows is None else rows
     cuq = np.concatenate([[0], np.cumsum(rows)]).astype(np.int32)
     q_idx = np.zeros(0, dtype=np.int32) if q_idx is None else np.asarray(q_idx, dtype=np.int32)
     clamped = [min(max(k, 0), n) for k, n in zip(keeps, lens)]
-    flags = (fastav.FASTAV_PROTECT_QUERY_ROWS if protect_rows else 0) | (fastav.FASTAV_KEEP_IDX_GLOBAL if global_idx else 0)
+    flags = ((fastav.FASTAV_PROTECT_QUERY_ROWS if protect_rows else 0) | (fastav.FASTAV_KEEP_IDX_GLOBAL if global_idx else 0) |
+             (fastav.FASTAV_SELECT_LOWEST if lowest else 0))
     params = fastav.make_params(batch=len(lens), total_tokens=int(cu[-1]), max_seqlen=max(lens), total_q=int(cuq[-1]),
                                 max_qlen=max(rows), total_keep=sum(clamped), max_keep=max(clamped), num_q_heads=4,
                                 num_kv_heads=2, head_dim=64, hidden=64, flags=flags)
@@ -173,7 +174,9 @@ def _select_case(lens, keeps, scores, protect=None, rows=None, q_idx=None, globa
                          None if protect is None else dev(protect, torch.uint8), dev(q_idx, torch.int32) if len(q_idx) else None,
                          dev(cuq, torch.int32), keep_idx, cu_keep, ws, status)
     torch.cuda.synchronize()
-    ref_idx, ref_cu = oracle.select(scores, cu, keeps, protect, protect_rows, q_idx, cuq, global_idx)
+    # keeping the lowest scores is keeping the highest of the negated scores (same tie rule)
+    ref_idx, ref_cu = oracle.select(-np.asarray(scores, dtype=np.float32) if lowest else scores, cu, keeps, protect, protect_rows,
+                                    q_idx, cuq, global_idx)
     assert cu_keep.cpu().tolist() == ref_cu.tolist()
     got = keep_idx.cpu().numpy()
     assert got[:len(ref_idx)].tolist() == ref_idx.tolist()
@@ -193,6 +196,15 @@ def test_select_matches_oracle_with_ties_protection_and_edge_sizes():
     assert _select_case(lens, keeps, scores, protect, global_idx=True) & ~fastav.FASTAV_DEV_PROTECT_OVERFLOW == 0
     smooth = rng.random(n).astype(np.float32) * 1e-3
     assert _select_case(lens, keeps, smooth) == 0
+
+
+def test_select_lowest_keeps_the_least_attended_tokens():
+    rng = np.random.default_rng(12)
+    lens, keeps = [700, 33, 4000], [300, 32, 1]
+    scores = (rng.integers(0, 200, size=sum(lens)) / 4096.0).astype(np.float32)
+    protect = (rng.random(sum(lens)) < 0.03).astype(np.uint8)
+    assert _select_case(lens, keeps, scores, lowest=True) == 0
+    assert _select_case(lens, keeps, scores, protect, lowest=True) & ~fastav.FASTAV_DEV_PROTECT_OVERFLOW == 0
 
 
 def test_select_general_floats_negative_zero_and_inf():
@@ -479,3 +491,22 @@ def test_prune_host_buffers_match_oracle():
     assert out["keep_idx"].tolist() == ref["keep_idx"].tolist()
     for name in ("hidden", "pos", "k", "v"):
         parity.assert_bits_equal(out[name], ref[name], "host " + name)
+
+
+def test_a_wait_that_cannot_succeed_ends_with_an_error_bit_and_a_usable_context():
+    """Failure detection without a fault: the kernels' waits are bounded; one that nothing satisfies gives up,
+    reports FASTAV_DEV_WAIT_EXPIRED, and the next call on the same context works."""
+    import time
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    fastav.fastav_selftest_bounded_wait(50, status)
+    torch.cuda.synchronize()
+    elapsed = time.perf_counter() - t0
+    assert int(status) == fastav.FASTAV_DEV_WAIT_EXPIRED
+    assert 0.04 < elapsed < 2.0
+    p = W.random_problem(seed=1, lens=[200], rows=[8], keeps=[100], num_q_heads=8, num_kv_heads=2, head_dim=64, hidden=64)
+    buf = parity.to_device(p)
+    buf.prune()
+    torch.cuda.synchronize()
+    parity.check_fused_against_oracle(p, buf, parity.oracle_prune(p), what="after the expired wait")
