@@ -248,7 +248,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="c4_long_av", choices=list(W.WORKLOAD_ORDER))
+    ap.add_argument("--workload", default="c4_long_av", choices=list(W.WORKLOAD_ORDER) + list(W.EXTRA_WORKLOADS))
+    ap.add_argument("--graph", action="store_true", help="also time the step replayed from a CUDA graph")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -318,6 +319,27 @@ def main():
                 step()
             torch.cuda.synchronize()
     barrier()
+    graph_replay = None
+    if args.graph:
+        # The whole step (every stage's kernel chain) captured once and replayed: no host launch cost per step.
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for _, buf in stages:
+                buf.prune(side)
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        ga, gb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ga.record()
+        for _ in range(args.steps):
+            graph.replay()
+        gb.record()
+        torch.cuda.synchronize()
+        graph_ms = R.max_over_ranks(ga.elapsed_time(gb) / args.steps, dist, device)
+        graph_replay = {"ms_per_step": graph_ms, "value": R.aggregate_throughput(tokens_per_step, graph_ms, world), "unit": "tokens/s",
+                        "note": "same kernels, enqueued by one graph launch; L2 not flushed between replays"}
     step_ms = [a.elapsed_time(b) for a, b in zip(starts, stops)]
     total_ms = sum(step_ms)
     total_ms = R.max_over_ranks(total_ms, dist, device)
@@ -427,7 +449,7 @@ def main():
             "step_hbm": {"algorithmic_bytes": bytes_per_step, "gbs": round(step_gbs, 1), "frac_of_peak": round(step_gbs / peaks["hbm_gbs"], 4),
                          "frac_of_nominal_8tbs": round(step_gbs / 8000.0, 4), "of": peaks["source"]},
             "roofline": roofline, "roofline_hbm": roofline_hbm, "compact_roofline": compact_rooflines, "phases": phases,
-            "prefill_flops": flops_removed(w, lens), "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": launches,
+            "prefill_flops": flops_removed(w, lens), "graph_replay": graph_replay, "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": launches,
             "device_status": status, "clocks": clocks.summary()}))
     if dist is not None:
         dist.destroy_process_group()

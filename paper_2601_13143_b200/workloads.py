@@ -81,9 +81,15 @@ WORKLOADS: dict[str, Workload] = {
         Workload("c5_ragged", 4, 4, QWEN2_7B, 32, (1024, 8192), None, 16,
                  (Stage(14, 32, None), Stage(15, 1, 0.8)), keep_range=(0.3, 0.7),
                  description="ragged serving batch, 32 sequences of 1024..8192 tokens, two stages"),
+        # Beyond the five configurations: the paper's own fine-pruning schedule on VideoLLaMA2-like sizes -- about 744
+        # survivors of the global stage (2,230 tokens, audio 1,496 -> 10), then P = 20 % at each of the 13 later layers.
+        Workload("n3_fine_chain_13", 5, 5, QWEN2_7B, 1, 744, None, 8,
+                 tuple(Stage(layer, 1, 0.8) for layer in range(15, 28)), sparse_positions=True,
+                 description="the paper's 13-layer fine-prune chain after the global stage, 744 -> ... -> 42, last-token query"),
     )
 }
 WORKLOAD_ORDER = ("c1_tiny", "c2_global_2k", "c3_fine_chain", "c4_long_av", "c5_ragged")
+EXTRA_WORKLOADS = ("n3_fine_chain_13",)
 
 
 def keep_count(n: int, keep_ratio: float) -> int:

@@ -117,6 +117,28 @@ def test_score_with_caller_provided_lse(lens, rows, hq, hkv, d, path):
     assert with_lse <= fastav.fastav_kernel_launches() - launches       # never more work than the self-contained path
 
 
+def test_score_many_sequences_and_one_very_long_sequence():
+    """More sequences than the tensor-core kernel has threads (its unit table is then walked serially), with empty
+    ones in between, and one sequence far longer than a block's share of key chunks."""
+    rng = np.random.default_rng(5)
+    lens = [int(x) for x in rng.integers(0, 40, size=700)]
+    rows = [min(n, int(r)) for n, r in zip(lens, rng.integers(5, 9, size=700))]
+    p = W.random_problem(seed=77, lens=lens, rows=rows, keeps=[n // 2 for n in lens], num_q_heads=4, num_kv_heads=2, head_dim=64,
+                         hidden=64)
+    for path in ("wide", "generic"):
+        buf = parity.to_device(p, extra_flags=SCORE_PATHS[path])
+        buf.score()
+        torch.cuda.synchronize()
+        assert int(buf.device_status.cpu()) == 0
+        parity.assert_scores_close(buf.scores, parity.oracle_scores(p), f"700 sequences, {path}")
+    p = W.random_problem(seed=78, lens=[70_001], rows=[6], keeps=[100], num_q_heads=4, num_kv_heads=1, head_dim=64, hidden=64)
+    buf = parity.to_device(p, extra_flags=SCORE_PATHS["wide"])
+    buf.score()
+    torch.cuda.synchronize()
+    assert int(buf.device_status.cpu()) == 0
+    parity.assert_scores_close(buf.scores, parity.oracle_scores(p), "one sequence of 70001 keys")
+
+
 def test_score_softmax_scale_one_is_eq4_as_printed():
     p = W.random_problem(seed=3, lens=[50], rows=[1], keeps=[25], num_q_heads=4, num_kv_heads=2, head_dim=64, hidden=64)
     p.softmax_scale = 1.0
@@ -455,7 +477,7 @@ def _run_workload_chain(name, stats_out=None):
         torch.cuda.empty_cache()
 
 
-@pytest.mark.parametrize("name", ["c1_tiny", "c2_global_2k", "c3_fine_chain"])
+@pytest.mark.parametrize("name", ["c1_tiny", "c2_global_2k", "c3_fine_chain", "n3_fine_chain_13"])
 def test_prune_workloads_small(name):
     _run_workload_chain(name)
 
