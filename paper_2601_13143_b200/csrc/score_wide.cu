@@ -13,20 +13,21 @@
 //            the block's query rows in a fixed column order; four such sums -> partial[KV head, row chunk][token];
 //   finalize: scores = (sum of the partials in a fixed order) / (Hq R).
 //
-// One block = one (sequence, KV head, chunk of 256 query rows, chunk of key tiles).  Warp 0 streams
-// 128-key K tiles with TMA (128-byte swizzle) through a 4-stage mbarrier ring, warp 1 issues the MMAs
-// into a double-buffered accumulator, warps 2-17 (four warpgroups) read the accumulators back with
-// tcgen05.ld and do the softmax arithmetic, part of the exponentials on the FMA pipe.  The per-key arithmetic does not depend on the key's
-// position, so equal keys get bit-equal scores; all sums have a fixed order, so runs are reproducible.
-// Every wait is bounded: a wait that expires makes the block give up, wait for its own copies, free its
-// tensor memory and set FASTAV_DEV_WAIT_EXPIRED.
+// One persistent block per SM works through its share of the units (sequence, KV head, chunk of up to 256
+// query rows, chunk of key tiles); the share is computed on the device from cu_seqlens.  Warp 0 streams
+// 128-key K tiles and the query tile with TMA (128-byte swizzle) through a 4-stage mbarrier ring, warp 1
+// issues the MMAs into double-buffered accumulators, warps 2-17 (four warpgroups) read the accumulators
+// back with tcgen05.ld and do the softmax arithmetic, part of the exponentials on the FMA pipe.  A third
+// mode of the same kernel only writes the scaled, masked logits (few scored rows: see score_narrow.cu).
+// The per-key arithmetic does not depend on the key's position, so equal keys get bit-equal scores; all
+// sums have a fixed order, so runs are reproducible.  Every wait is bounded: a wait that expires makes the
+// block give up, wait for its own copies, free its tensor memory and set FASTAV_DEV_WAIT_EXPIRED.
 #include <cuda.h>
 
 #include <limits.h>
 
 #include "common.cuh"
 #include "sm100_ptx.cuh"
-
 
 namespace fastav {
 namespace {
