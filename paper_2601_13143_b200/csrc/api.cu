@@ -272,10 +272,19 @@ int32_t fastav_prune(const fastav_params* params, const void* q, const int32_t* 
   unsigned char* ws = static_cast<unsigned char*>(workspace);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e = cudaSuccess;
-  if (params->total_tokens > 0) e = launch_score(s, w, q, q_idx, cu_qlens, k, cu_seqlens, nullptr, scores_out, ws, device_status, st);
-  if (e == cudaSuccess)
-    e = launch_select(s, w, scores_out, cu_seqlens, keep_counts, protect_opt, q_idx, cu_qlens, keep_idx_out, cu_keep_out, ws,
-                      device_status, st);
+  const unsigned forced = s.flags & FASTAV_SCORE_PATH_MASK;
+  if (params->total_tokens > 0 && score_narrow_applies(s) && narrow_tail_applies(s) && (forced == 0 || forced == FASTAV_SCORE_PATH_NARROW)) {
+    // Short sequences, few scored rows: logits, then ONE kernel for the softmax statistics, the scores and the keep list.
+    e = launch_narrow_logits(s, w, q, q_idx, cu_qlens, k, cu_seqlens, ws, device_status, st);
+    if (e == cudaSuccess)
+      e = launch_narrow_tail(s, reinterpret_cast<const float*>(ws + w.logits_off), s.max_qlen, scores_out, true, cu_seqlens,
+                             keep_counts, protect_opt, q_idx, cu_qlens, keep_idx_out, cu_keep_out, device_status, st);
+  } else {
+    if (params->total_tokens > 0) e = launch_score(s, w, q, q_idx, cu_qlens, k, cu_seqlens, nullptr, scores_out, ws, device_status, st);
+    if (e == cudaSuccess)
+      e = launch_select(s, w, scores_out, cu_seqlens, keep_counts, protect_opt, q_idx, cu_qlens, keep_idx_out, cu_keep_out, ws,
+                        device_status, st);
+  }
   if (e == cudaSuccess)
     e = launch_compact(s, keep_idx_out, cu_keep_out, cu_seqlens, hidden_in, hidden_out, pos_in, pos_out, k, k_out, v, v_out,
                        device_status, st);

@@ -71,6 +71,17 @@ cudaError_t launch_logits_wide(const Shapes& s, const void* q, const int32_t* q_
                                const int32_t* cu_seqlens, float* logits, int rq, int32_t* device_status, cudaStream_t stream,
                                bool* used);
 
+// Short sequences with few scored rows: one kernel turns the logits into scores and (optionally) the keep list.
+bool narrow_tail_applies(const Shapes& s);
+cudaError_t launch_narrow_tail(const Shapes& s, const float* logits, int rq, float* scores_out, bool do_select,
+                               const int32_t* cu_seqlens, const int32_t* keep_counts, const uint8_t* protect,
+                               const int32_t* q_idx, const int32_t* cu_qlens, int32_t* keep_idx, int32_t* cu_keep,
+                               int32_t* device_status, cudaStream_t stream);
+// Only the logits [Hq, max_qlen, N] of the few-rows path, into the workspace.
+cudaError_t launch_narrow_logits(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
+                                 const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, unsigned char* ws,
+                                 int32_t* device_status, cudaStream_t stream);
+
 cudaError_t launch_select(const Shapes& s, const Workspace& w, const float* scores, const int32_t* cu_seqlens,
                           const int32_t* keep_counts, const uint8_t* protect, const int32_t* q_idx,
                           const int32_t* cu_qlens, int32_t* keep_idx, int32_t* cu_keep, unsigned char* ws,

@@ -310,13 +310,12 @@ cudaError_t launch_logits(const Shapes& s, const uint16_t* q, const int32_t* q_i
 
 bool score_narrow_applies(const Shapes& s) { return s.max_qlen >= 1 && s.max_qlen <= kNarrowMaxRows && s.hq <= 256; }
 
-cudaError_t launch_score_narrow(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
-                                const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, const float* lse_in,
-                                float* scores_out, unsigned char* ws, int32_t* device_status, cudaStream_t stream) {
+cudaError_t launch_narrow_logits(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
+                                 const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, unsigned char* ws,
+                                 int32_t* device_status, cudaStream_t stream) {
   const uint16_t* qq = static_cast<const uint16_t*>(q);
   const uint16_t* kk = static_cast<const uint16_t*>(k);
   float* logits = reinterpret_cast<float*>(ws + w.logits_off);
-  float* lse = reinterpret_cast<float*>(ws + w.lse_off);
   const int rq = s.max_qlen;
   const bool four = s.max_qlen * s.group <= 4;
   cudaError_t e;
@@ -325,18 +324,30 @@ cudaError_t launch_score_narrow(const Shapes& s, const Workspace& w, const void*
   bool by_mma = false;
   if ((s.flags & FASTAV_SCORE_PATH_MASK) != FASTAV_SCORE_PATH_NARROW && score_wide_applies(s)) {
     e = launch_logits_wide(s, q, q_idx, cu_qlens, k, cu_seqlens, logits, rq, device_status, stream, &by_mma);
-    if (e != cudaSuccess) return e;
+    if (e != cudaSuccess || by_mma) return e;
   }
-  if (by_mma) {
-    e = cudaSuccess;
-  } else if (s.dim == 128) {
+  if (s.dim == 128) {
     e = four ? launch_logits<128, 4>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, device_status, stream)
              : launch_logits<128, 8>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, device_status, stream);
   } else {
     e = four ? launch_logits<64, 4>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, device_status, stream)
              : launch_logits<64, 8>(s, qq, q_idx, cu_qlens, kk, cu_seqlens, logits, rq, device_status, stream);
   }
+  count_launches(1);
+  return e;
+}
+
+cudaError_t launch_score_narrow(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,
+                                const int32_t* cu_qlens, const void* k, const int32_t* cu_seqlens, const float* lse_in,
+                                float* scores_out, unsigned char* ws, int32_t* device_status, cudaStream_t stream) {
+  float* logits = reinterpret_cast<float*>(ws + w.logits_off);
+  float* lse = reinterpret_cast<float*>(ws + w.lse_off);
+  const int rq = s.max_qlen;
+  cudaError_t e = launch_narrow_logits(s, w, q, q_idx, cu_qlens, k, cu_seqlens, ws, device_status, stream);
   if (e != cudaSuccess) return e;
+  if (!lse_in && narrow_tail_applies(s))  // short sequences: statistics and scores in one kernel
+    return launch_narrow_tail(s, logits, rq, scores_out, false, cu_seqlens, nullptr, nullptr, q_idx, cu_qlens, nullptr, nullptr,
+                              device_status, stream);
   if (lse_in) e = launch_lse_import(s, lse_in, lse, stream);
   else e = launch_chained(score_narrow_stats_kernel, dim3(s.hq * rq, s.batch), dim3(256), 0, stream, s, cu_qlens, cu_seqlens,
                           (const float*)logits, rq, lse);
@@ -346,7 +357,7 @@ cudaError_t launch_score_narrow(const Shapes& s, const Workspace& w, const void*
                           s.hq * rq * sizeof(float), stream, s, cu_qlens, cu_seqlens, (const float*)logits, rq, (const float*)lse,
                           scores_out)) != cudaSuccess)
     return e;
-  count_launches((by_mma ? 0 : 1) + (lse_in ? 0 : 1) + 1);  // the tensor-core logits and the lse import count themselves
+  count_launches((lse_in ? 0 : 1) + 1);  // the lse import counts itself
   return cudaGetLastError();
 }
 

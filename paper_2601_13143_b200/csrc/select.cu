@@ -45,7 +45,18 @@ struct SelectShared {
 template <bool kKeysInShared>
 __device__ __forceinline__ int slot(int j) { return kKeysInShared ? j + (j >> 5) : j; }
 
-template <bool kKeysInShared>
+// Few scored rows, short sequences: the scores themselves are made here, from the logits the previous
+// kernel left in the workspace (one block per sequence: log2-sum-exp2 per (head, row) by one warp each,
+// then per token the fixed-order sum over heads and rows), so that a pruning layer of a small prompt is
+// three kernels (logits, this one, the gather) instead of five.
+struct FromLogits {
+  const float* logits;  // [Hq, rq, N] base-2 logits, -inf where masked
+  float* scores_out;    // [N]
+  int rq;               // scored rows per sequence the logits are laid out for
+  int do_select;        // 0: only the scores are wanted (fastav_score)
+};
+
+template <bool kKeysInShared, bool kFromLogits>
 __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const float* __restrict__ scores,
                                                                const int32_t* __restrict__ cu_seqlens,
                                                                const int32_t* __restrict__ keep_counts,
@@ -53,7 +64,8 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
                                                                const int32_t* __restrict__ q_idx,
                                                                const int32_t* __restrict__ cu_qlens,
                                                                int32_t* __restrict__ keep_idx, int32_t* __restrict__ cu_keep,
-                                                               unsigned* __restrict__ keys_global, int32_t* device_status) {
+                                                               unsigned* __restrict__ keys_global, int32_t* device_status,
+                                                               FromLogits fl) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   SelectShared& sh = *reinterpret_cast<SelectShared*>(smem_raw);
   unsigned* keys = kKeysInShared ? reinterpret_cast<unsigned*>(smem_raw + sizeof(SelectShared)) : nullptr;
@@ -63,10 +75,11 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
   const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
   if (!kKeysInShared) keys = keys_global + tok0;
 
+  const bool selecting = !kFromLogits || fl.do_select != 0;
   // Output offset: prefix sum of the clamped keep counts of the sequences before this one.
   if (tid == 0) { sh.base = 0; sh.protected_count = 0; sh.key_min = 0xFFFFFFFFu; sh.key_max = 0u; }
   __syncthreads();
-  {
+  if (selecting) {
     int part = 0;
     bool clamped = false;
     for (int i = tid; i <= b; i += kThreads) {
@@ -78,14 +91,67 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
     if (part) atomicAdd(&sh.base, part);
     if (clamped && device_status) atomicOr(device_status, FASTAV_DEV_K_CLAMPED);
   }
-  int k = keep_counts[b];
+  int k = selecting ? keep_counts[b] : 0;
   k = k < 0 ? 0 : (k > n ? n : k);
 
-  pdl_wait();  // the scores are the previous kernel's output
+  pdl_wait();  // the scores (or logits) are the previous kernel's output
   pdl_acquire(scores);
 
   // Keys.  Under FASTAV_SELECT_LOWEST the ranking is reversed by negating the scores (ties still go to the lower index).
   const bool lowest = (s.flags & FASTAV_SELECT_LOWEST) != 0;
+  if constexpr (kFromLogits) {
+    pdl_acquire(fl.logits);
+    float* lse_sh = reinterpret_cast<float*>(keys + (s.max_seqlen + s.max_seqlen / 32 + 1));
+    const int row0 = cu_qlens[b], all_rows = cu_qlens[b + 1] - row0, rows = min(all_rows, fl.rq);
+    const int terms = s.hq * rows;  // term i = (head i / rows, row i % rows)
+    for (int i = warp; i < terms; i += kWarps) {
+      // log2-sum-exp2 of one row of logits by one warp: running (max, sum) per lane, merged in a fixed order
+      const float* z = fl.logits + ((long long)(i / rows) * fl.rq + i % rows) * s.total_tokens + tok0;
+      float m = -INFINITY, l = 0.f;
+      for (int j0 = lane; j0 < n; j0 += 128) {
+        float v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = j0 + 32 * u < n ? z[j0 + 32 * u] : -INFINITY;
+        const float m_new = fmaxf(fmaxf(m, fmaxf(v[0], v[1])), fmaxf(v[2], v[3]));
+        if (m_new > -INFINITY) {
+          l = l * exp2f(m - m_new);
+#pragma unroll
+          for (int u = 0; u < 4; ++u) l += exp2f(v[u] - m_new);
+          m = m_new;
+        }
+      }
+      float bm = m;
+#pragma unroll
+      for (int d = 16; d; d >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xFFFFFFFFu, bm, d));
+      float part = (m > -INFINITY) ? l * exp2f(m - bm) : 0.f;
+#pragma unroll
+      for (int d = 16; d; d >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, d);
+      if (lane == 0) lse_sh[i] = part > 0.f ? bm + log2f(part) : INFINITY;  // a row that sees no key adds 0
+    }
+    __syncthreads();
+    for (int j = tid; j < n; j += kThreads) {
+      const float* z = fl.logits + tok0 + j;
+      float total = 0.f;
+      for (int i0 = 0; i0 < terms; i0 += 8) {
+        float v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int i = i0 + u;
+          v[u] = i < terms ? z[((long long)(i / rows) * fl.rq + i % rows) * s.total_tokens] : -INFINITY;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+          if (i0 + u < terms) total += exp2f(v[u] - lse_sh[i0 + u]);
+      }
+      const float score = all_rows > 0 ? total / ((float)s.hq * (float)all_rows) : 0.f;
+      fl.scores_out[tok0 + j] = score;
+      unsigned key = order_key(lowest ? -score : score);
+      if (key == kProtectedKey) key = kProtectedKey - 1;
+      if (protect && protect[tok0 + j]) key = kProtectedKey;
+      keys[slot<kKeysInShared>(j)] = key;
+    }
+    if (!selecting) return;  // uniform for the block
+  } else
   for (int j0 = tid; j0 < n; j0 += kThreads * 16) {
     float v[16];  // sixteen independent loads in flight per thread: one block serves a whole sequence
 #pragma unroll
@@ -265,14 +331,39 @@ cudaError_t launch_select(const Shapes& s, const Workspace& w, const float* scor
   constexpr size_t kMaxDynamic = 227 * 1024 - 1024;
   cudaError_t e;
   if (want <= kMaxDynamic) {
-    e = cudaFuncSetAttribute(select_topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynamic);
+    e = cudaFuncSetAttribute(select_topk_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynamic);
     if (e != cudaSuccess) return e;
-    e = launch_chained(select_topk_kernel<true>, dim3(s.batch), dim3(kThreads), want, stream, s, scores, cu_seqlens, keep_counts,
-                       protect, q_idx, cu_qlens, keep_idx, cu_keep, (unsigned*)nullptr, device_status);
+    e = launch_chained(select_topk_kernel<true, false>, dim3(s.batch), dim3(kThreads), want, stream, s, scores, cu_seqlens,
+                       keep_counts, protect, q_idx, cu_qlens, keep_idx, cu_keep, (unsigned*)nullptr, device_status, FromLogits{});
   } else {
-    e = launch_chained(select_topk_kernel<false>, dim3(s.batch), dim3(kThreads), fixed, stream, s, scores, cu_seqlens, keep_counts,
-                       protect, q_idx, cu_qlens, keep_idx, cu_keep, reinterpret_cast<unsigned*>(ws + w.keys_off), device_status);
+    e = launch_chained(select_topk_kernel<false, false>, dim3(s.batch), dim3(kThreads), fixed, stream, s, scores, cu_seqlens,
+                       keep_counts, protect, q_idx, cu_qlens, keep_idx, cu_keep, reinterpret_cast<unsigned*>(ws + w.keys_off),
+                       device_status, FromLogits{});
   }
+  count_launches(1);
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+// Scores (and, with `do_select`, the keep list) of a batch of short sequences with few scored rows, straight
+// from the logits in the workspace.
+bool narrow_tail_applies(const Shapes& s) {
+  const size_t smem = sizeof(SelectShared) + ((size_t)s.max_seqlen + s.max_seqlen / 32 + 1) * sizeof(unsigned) +
+                      (size_t)s.hq * s.max_qlen * sizeof(float);
+  // one block per sequence does all of it: worth it only while a sequence is short (measured: up to about 1k tokens)
+  return s.max_qlen >= 1 && s.max_qlen <= kNarrowMaxRows && s.max_seqlen >= 1 && s.max_seqlen <= 1024 && smem <= 200 * 1024;
+}
+
+cudaError_t launch_narrow_tail(const Shapes& s, const float* logits, int rq, float* scores_out, bool do_select,
+                               const int32_t* cu_seqlens, const int32_t* keep_counts, const uint8_t* protect,
+                               const int32_t* q_idx, const int32_t* cu_qlens, int32_t* keep_idx, int32_t* cu_keep,
+                               int32_t* device_status, cudaStream_t stream) {
+  const size_t smem = sizeof(SelectShared) + ((size_t)s.max_seqlen + s.max_seqlen / 32 + 1) * sizeof(unsigned) +
+                      (size_t)s.hq * rq * sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(select_topk_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  if (e != cudaSuccess) return e;
+  e = launch_chained(select_topk_kernel<true, true>, dim3(s.batch), dim3(kThreads), smem, stream, s, (const float*)nullptr,
+                     cu_seqlens, keep_counts, protect, q_idx, cu_qlens, keep_idx, cu_keep, (unsigned*)nullptr, device_status,
+                     FromLogits{logits, scores_out, rq, do_select ? 1 : 0});
   count_launches(1);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -431,8 +522,8 @@ extern "C" int32_t fastav_select_noalloc(const fastav_params* p, const float* sc
   s.flags = p->flags;
   // Every key a block reads was written by that block earlier in the same launch, so what an
   // earlier call left in the array never matters and nothing has to be cleared.
-  select_topk_kernel<false><<<s.batch, kThreads, sizeof(SelectShared), static_cast<cudaStream_t>(stream)>>>(
-      s, scores, cu_seqlens, keep_counts, protect_opt, q_idx, cu_qlens, keep_idx_out, cu_keep_out, keys, device_status);
+  select_topk_kernel<false, false><<<s.batch, kThreads, sizeof(SelectShared), static_cast<cudaStream_t>(stream)>>>(
+      s, scores, cu_seqlens, keep_counts, protect_opt, q_idx, cu_qlens, keep_idx_out, cu_keep_out, keys, device_status, FromLogits{});
   count_launches(1);
   return cudaGetLastError() == cudaSuccess ? FASTAV_OK : FASTAV_ERR_CUDA;
 }
