@@ -38,6 +38,10 @@ constexpr int kStages = 4;        // K tiles in flight
 constexpr int kGroups = 4;        // softmax warpgroups: four warps per scheduler hide each other's latencies
 constexpr int kThreads = 64 + 128 * kGroups;  // warp 0: TMA, warp 1: MMA, warps 2-17: softmax
 constexpr int kTmemCols = 512;
+#ifndef FASTAV_UNITS_PER_BLOCK
+#define FASTAV_UNITS_PER_BLOCK 7
+#endif
+constexpr int kUnitsPerBlock = FASTAV_UNITS_PER_BLOCK;  // aimed-at number of work units per block
 constexpr int kMaxUnits = 48;       // work units one block may be given (the host sizes key chunks accordingly)
 constexpr int kCtrlBytes = 18 * 1024;
 
@@ -81,7 +85,7 @@ __device__ __forceinline__ float2 exp2_pair_fma(float2 x) {
 // The softmax is bound by exponentials, so they are split over two pipes: of the 8 column pairs of every
 // 16-column block, the pairs in kFmaPairs go through exp2_pair_fma, the others through the special-function unit.
 #ifndef FASTAV_FMA_PAIRS
-#define FASTAV_FMA_PAIRS 0x92  // pairs 1, 4, 7: three of eight
+#define FASTAV_FMA_PAIRS 0x88  // pairs 3 and 7: two of eight (three or four of eight measured no faster)
 #endif
 constexpr unsigned kFmaPairs = FASTAV_FMA_PAIRS;
 
@@ -782,7 +786,7 @@ void plan_units(const Shapes& s, int rc_max, int* grid_out, int* chunk_tiles_out
   const long long tiles_upper = (long long)s.total_tokens / kTileKeys + s.batch;  // >= sum over sequences of ceil(n / 128)
   const long long tile_units = tiles_upper * s.hkv * rc_max;
   const int grid = (int)(tile_units < kNumSMs ? tile_units : kNumSMs);
-  long long chunk_tiles = (tile_units + (long long)grid * 14 - 1) / ((long long)grid * 14);
+  long long chunk_tiles = (tile_units + (long long)grid * kUnitsPerBlock - 1) / ((long long)grid * kUnitsPerBlock);
   if (chunk_tiles < 1) chunk_tiles = 1;
   // units <= hkv * rc_max * (tokens / chunk + batch); keep the per-block share within the table
   while (((long long)s.hkv * rc_max * (s.total_tokens / (chunk_tiles * kTileKeys) + s.batch) + grid - 1) / grid + 1 > kMaxUnits)
