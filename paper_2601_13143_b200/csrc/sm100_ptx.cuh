@@ -40,11 +40,30 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// The same with a suspend-time hint: the thread may sleep in hardware for up to `hint_ns` (it is woken when
+// the phase completes), so a waiting warp does not burn issue slots the working warps need.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(hint_ns)
+      : "memory");
+  return ok != 0;
+}
 
 // Waits for the phase with the given parity to complete, but never for ever: gives up when `*abort`
 // becomes non-zero (another thread of the block gave up) or after kWaitLimitNs, in which case it sets
 // `*abort` itself.  Returns false when it gave up.
 constexpr uint64_t kWaitLimitNs = 500ull * 1000 * 1000;
+#ifndef FASTAV_SUSPEND_HINT_NS
+#define FASTAV_SUSPEND_HINT_NS 2000
+#endif
+constexpr uint32_t kSuspendHintNs = FASTAV_SUSPEND_HINT_NS;
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort,
                                                   uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
@@ -53,7 +72,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
     // a short tight run of attempts (each may suspend the thread for a while in hardware), then the checks
 #pragma unroll 1
     for (int i = 0; i < 16; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
+      if (mbar_try_wait_hint(bar, parity, kSuspendHintNs)) return true;
     if (*abort) return false;
     if (global_timer_ns() - t0 > limit_ns) {
       *abort = 1;
