@@ -176,6 +176,60 @@ def run_host_step(chain):
                                  h["pos_out"], h["k_out"], h["v_out"], h["status"], h["arena"])
 
 
+def host_chain_per_sequence(w: W.Workload, device, n_streams: int = 2):
+    """The same pinned host tensors cut into one prune_host call per (sequence, stage), the sequences dealt over
+    ``n_streams`` CUDA streams: the upload of one sequence overlaps the kernels and the download of another (PCIe is
+    full duplex), which a single call on a single stream cannot do.  Returns (calls per stream, streams, chain)."""
+    from paper_2601_13143_b200 import fastav
+    chain = host_chain(w, device)
+    pin = lambda t: t.contiguous().pin_memory()
+    i32 = lambda xs: pin(torch.tensor(xs, dtype=torch.int32))
+    streams = [torch.cuda.Stream(device=device) for _ in range(n_streams)]
+    arena_bytes = [0] * n_streams
+    calls = [[] for _ in range(n_streams)]
+    for b in range(w.batch):
+        slot = b % n_streams
+        for si, h in enumerate(chain):
+            p = W.make_stage(w, si)
+            m = p.model
+            cu, cuq = p.cu_seqlens.tolist(), p.cu_qlens.tolist()
+            keeps = p.keep_counts.tolist()
+            cuk = [0]
+            for kb in keeps:
+                cuk.append(cuk[-1] + kb)
+            n, r, kb = cu[b + 1] - cu[b], cuq[b + 1] - cuq[b], keeps[b]
+            params = fastav.make_params(batch=1, total_tokens=n, max_seqlen=n, total_q=r, max_qlen=r, total_keep=kb, max_keep=kb,
+                                        num_q_heads=m.num_q_heads, num_kv_heads=m.num_kv_heads, head_dim=m.head_dim,
+                                        hidden=m.hidden, softmax_scale=p.softmax_scale,
+                                        flags=fastav.FASTAV_CAUSAL | fastav.FASTAV_PROTECT_QUERY_ROWS)
+            tok, row, out = slice(cu[b], cu[b + 1]), slice(cuq[b], cuq[b + 1]), slice(cuk[b], cuk[b + 1])
+            c = {"params": params, "q": h["q"][row], "q_idx": h["q_idx"][row], "cu_qlens": i32([0, r]), "k": h["k"][tok], "v": h["v"][tok],
+                 "cu_seqlens": i32([0, n]), "keep_counts": i32([kb]), "hidden": h["hidden"][tok], "pos": h["pos"][tok],
+                 "scores": h["scores"][tok], "keep_idx": h["keep_idx"][out], "cu_keep": pin(torch.empty(2, dtype=torch.int32)),
+                 "hidden_out": h["hidden_out"][out], "pos_out": h["pos_out"][out], "k_out": h["k_out"][out], "v_out": h["v_out"][out],
+                 "status": pin(torch.zeros(1, dtype=torch.int32))}
+            arena_bytes[slot] = max(arena_bytes[slot], fastav.fastav_host_arena_bytes(params))
+            calls[slot].append(c)
+    arenas = [torch.empty(max(nb, 256), dtype=torch.uint8, device=device) for nb in arena_bytes]
+    for slot in range(n_streams):
+        for c in calls[slot]:
+            c["arena"] = arenas[slot]
+    return calls, streams, chain
+
+
+def run_host_step_per_sequence(calls, streams, main_stream):
+    from paper_2601_13143_b200 import fastav
+    start = torch.cuda.Event()
+    start.record(main_stream)
+    for st, mine in zip(streams, calls):
+        st.wait_event(start)
+        for c in mine:
+            fastav.fastav_prune_host(c["params"], c["q"], c["q_idx"], c["cu_qlens"], c["k"], c["v"], c["cu_seqlens"], c["keep_counts"],
+                                     None, c["hidden"], c["pos"], c["scores"], c["keep_idx"], c["cu_keep"], c["hidden_out"],
+                                     c["pos_out"], c["k_out"], c["v_out"], c["status"], c["arena"], stream=st)
+        main_stream.wait_stream(st)
+
+
 def oracle_sample(w: W.Workload):
     """Bounded sample for the CPU legs: the first sequence of every stage."""
     sys.path.insert(0, os.path.join(ROOT, "tests"))
@@ -406,23 +460,29 @@ def main():
     # ---- end to end: host buffers through fastav_prune_host, copies inside the timed region ----
     e2e = None
     if not args.no_e2e:
-        chain = host_chain(w, device)
         e2e_steps = min(args.steps, 5)
-        run_host_step(chain)
+        if w.batch > 1:  # one call per sequence and stage, two streams: uploads, kernels and downloads of different sequences overlap
+            calls, e2e_streams, chain = host_chain_per_sequence(w, device)
+            one_step = lambda: run_host_step_per_sequence(calls, e2e_streams, stream)
+            api = "fastav_prune_host, one call per sequence and stage on 2 streams (pinned host buffers)"
+        else:
+            chain = host_chain(w, device)
+            one_step = lambda: run_host_step(chain)
+            api = "fastav_prune_host (pinned host buffers)"
+        one_step()
         torch.cuda.synchronize()
         barrier()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(stream)
         for _ in range(e2e_steps):
-            run_host_step(chain)
+            one_step()
         b.record(stream)
         torch.cuda.synchronize()
         barrier()
         e2e_ms = a.elapsed_time(b) / e2e_steps
         e2e_ms = R.max_over_ranks(e2e_ms, dist, device)
         e2e = {"value": R.aggregate_throughput(tokens_per_step, e2e_ms, world), "unit": "tokens/s", "ms_per_step": e2e_ms, "steps": e2e_steps,
-               "h2d_bytes_per_step": sum(h["h2d"] for h in chain), "d2h_bytes_per_step": sum(h["d2h"] for h in chain),
-               "api": "fastav_prune_host (pinned host buffers)"}
+               "h2d_bytes_per_step": sum(h["h2d"] for h in chain), "d2h_bytes_per_step": sum(h["d2h"] for h in chain), "api": api}
         del chain
 
     cpu = None

@@ -526,3 +526,29 @@ def test_a_wait_that_cannot_succeed_ends_with_an_error_bit_and_a_usable_context(
     buf.prune()
     torch.cuda.synchronize()
     parity.check_fused_against_oracle(p, buf, parity.oracle_prune(p), what="after the expired wait")
+
+
+def test_bench_per_sequence_host_pipeline_equals_one_batched_call():
+    """bench.py's end-to-end leg cuts a batch into one host-buffer call per sequence and stage on two streams;
+    every output must equal what the single batched call writes."""
+    import os, sys
+    sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+    import bench
+    w = W.Workload("mini_ragged", 9, 9, W.TINY, 3, (200, 600), None, 4, (W.Stage(2, 5, None), W.Stage(3, 1, 0.8)),
+                   keep_range=(0.3, 0.7), description="test only")
+    dev = torch.device("cuda", 0)
+    chain = bench.host_chain(w, dev)
+    bench.run_host_step(chain)
+    torch.cuda.synchronize()
+    names = ("scores", "keep_idx", "hidden_out", "pos_out", "k_out", "v_out")
+    want = [{k: h[k].clone() for k in names} for h in chain]
+    calls, streams, chain2 = bench.host_chain_per_sequence(w, dev)
+    for h in chain2:
+        for k in names:
+            h[k].view(torch.uint8).fill_(0xEE)
+    bench.run_host_step_per_sequence(calls, streams, torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    for si, h in enumerate(chain2):
+        for k in names:
+            assert torch.equal(h[k].view(torch.uint8), want[si][k].view(torch.uint8)), (si, k)
+    assert all(int(c["status"]) == 0 for mine in calls for c in mine)
