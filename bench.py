@@ -230,6 +230,25 @@ def run_host_step_per_sequence(calls, streams, main_stream):
         main_stream.wait_stream(st)
 
 
+def attention_lse(p, buf) -> torch.Tensor:
+    """Natural-log log-sum-exp per (scored row, head) over the keys the row sees: the by-product an attention kernel
+    returns for these rows, made here with torch on the device (an INPUT of the secondary measurement only)."""
+    hq, hkv = buf.q.shape[1], buf.k.shape[1]
+    out = torch.empty((buf.q.shape[0], hq), dtype=torch.float32, device=buf.q.device)
+    cu, cuq = p.cu_seqlens.tolist(), p.cu_qlens.tolist()
+    for b in range(len(cu) - 1):
+        if cuq[b + 1] == cuq[b] or cu[b + 1] == cu[b]:
+            continue
+        k = buf.k[cu[b]:cu[b + 1]].float()                                                # [n, Hkv, d]
+        q = buf.q[cuq[b]:cuq[b + 1]].float().view(-1, hkv, hq // hkv, buf.q.shape[2])         # [R, Hkv, G, d]
+        z = torch.einsum("rgcd,ngd->rgcn", q, k) * p.softmax_scale                          # [R, Hkv, G, n]
+        if p.causal:
+            visible = torch.arange(k.shape[0], device=k.device)[None, :] <= buf.q_idx[cuq[b]:cuq[b + 1]][:, None]
+            z = z.masked_fill(~visible[:, None, None, :], float("-inf"))
+        out[cuq[b]:cuq[b + 1]] = torch.logsumexp(z, dim=-1).reshape(-1, hq)
+    return out
+
+
 def oracle_sample(w: W.Workload):
     """Bounded sample for the CPU legs: the first sequence of every stage."""
     sys.path.insert(0, os.path.join(ROOT, "tests"))
@@ -416,6 +435,25 @@ def main():
             for j, name in enumerate(("score", "select", "compact")):
                 phase_ms[si][name] += ev[j].elapsed_time(ev[j + 1]) / reps
 
+    # ---- secondary line: the score when the caller hands over the attention kernel's log-sum-exp (one sweep) ----
+    lse_ms = [None] * len(stages)
+    for si, (p, buf) in enumerate(stages):
+        if int((p.cu_qlens[1:] - p.cu_qlens[:-1]).max()) <= 4:
+            continue  # few scored rows: the statistics are a small part of that path
+        lse = attention_lse(p, buf)
+        for i in range(3 + reps):
+            if flush_buf is not None:
+                flush_buf.fill_(i & 0xFF)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fastav.fastav_score(buf.params, buf.q, buf.q_idx, buf.cu_qlens, buf.k, buf.cu_seqlens, buf.scores, buf.workspace,
+                                buf.device_status, stream, lse_opt=lse)
+            b.record(stream)
+            torch.cuda.synchronize()
+            if i >= 3:
+                lse_ms[si] = (lse_ms[si] or 0.0) + a.elapsed_time(b) / reps
+        del lse
+
     peaks = measured_peaks()
     phases = []
     for si, ((p, _), b, t) in enumerate(zip(stages, bytes_per_stage, phase_ms)):
@@ -423,7 +461,8 @@ def main():
                                 for i in range(p.batch)) * p.model.num_q_heads
         phases.append({"stage": si, "tokens": p.total_tokens, "ms": {k: round(v, 5) for k, v in t.items()},
                        "gbs": {k: round(b[k] / (t[k] * 1e-3) / 1e9, 1) if t[k] > 0 else None for k in t},
-                       "bytes": b, "score_exp2_per_sweep": rows_heads_tokens})
+                       "bytes": b, "score_exp2_per_sweep": rows_heads_tokens,
+                       "score_ms_given_attention_lse": None if lse_ms[si] is None else round(lse_ms[si], 5)})
     # ---- rooflines.  Which bound applies depends on the kernel:
     #   compact, select, matrix-vector score: HBM bytes (algorithmic bytes / time vs the measured copy peak);
     #   tensor-core score (many scored rows): the exponentials of the two softmax sweeps -- its K traffic is a small
