@@ -552,3 +552,35 @@ def test_bench_per_sequence_host_pipeline_equals_one_batched_call():
         for k in names:
             assert torch.equal(h[k].view(torch.uint8), want[si][k].view(torch.uint8)), (si, k)
     assert all(int(c["status"]) == 0 for mine in calls for c in mine)
+
+
+@pytest.mark.parametrize("lens,rows,hq,hkv,d", [([1500, 300], [64, 40], 8, 2, 128), ([900], [2], 28, 4, 128), ([400, 77], [9, 5], 4, 4, 64)])
+@pytest.mark.parametrize("path", ["auto", "generic", "narrow"])
+def test_workspace_guard_band_and_equal_keys_tie_bit_exactly(lens, rows, hq, hkv, d, path):
+    """(1) Nothing is written past fastav_workspace_bytes: a sentinel band after the workspace survives a fused call.
+    (2) The per-key arithmetic does not depend on the key's position: with every row seeing every key, tokens that
+    carry the same key vector get bit-equal scores."""
+    if path == "narrow" and max(rows) > 4:
+        pytest.skip("path does not take these shapes")
+    p = W.random_problem(seed=3, lens=lens, rows=rows, keeps=[n // 3 for n in lens], num_q_heads=hq, num_kv_heads=hkv, head_dim=d,
+                         hidden=64)
+    p.causal = False
+    cu = p.cu_seqlens.tolist()
+    twins = []
+    for b in range(len(lens)):            # copy token 5 of each sequence over a few other tokens, far apart
+        for j in (17, lens[b] // 2, lens[b] - 1):
+            p.k[cu[b] + j] = p.k[cu[b] + 5]
+            twins.append((cu[b] + 5, cu[b] + j))
+    buf = parity.to_device(p, extra_flags=SCORE_PATHS[path])
+    need = fastav.fastav_workspace_bytes(buf.params)
+    guard = 4096
+    ws = torch.full((need + guard,), 0x5A, dtype=torch.uint8, device="cuda")
+    buf.workspace = ws[:need]
+    buf.prune()
+    torch.cuda.synchronize()
+    assert int(buf.device_status.cpu()) == 0
+    assert bool((ws[need:] == 0x5A).all()), "the workspace was overrun"
+    parity.assert_scores_close(buf.scores, parity.oracle_scores(p), "guarded call")
+    bits = buf.scores.view(torch.int32).cpu()
+    for a, b in twins:
+        assert int(bits[a]) == int(bits[b]), (a, b)
