@@ -254,6 +254,29 @@ def test_select_sequence_longer_than_shared_memory():
     assert _select_case([n, 100], [n // 3, 50], scores=np.concatenate([scores, rng.random(100).astype(np.float32)])) == 0
 
 
+@pytest.mark.parametrize("longest", [2048, 2049, 4097, 8200, 16384, 40_000, 131_072, 131_073])
+def test_select_long_sequences_in_ragged_batches(longest):
+    """Keep lists of long sequences (keys in shared memory up to about 57k tokens, in the workspace above)
+    with short and empty sequences in the same batch: heavy ties, protected tokens and scored rows anywhere,
+    a long run of equal scores, nearly everything or nearly nothing kept."""
+    rng = np.random.default_rng(longest)
+    lens = [longest, 0, 1, 33, longest // 3, 1000]
+    keeps = [longest // 2, 0, 1, 20, longest // 3 - 1, 1]
+    n = sum(lens)
+    scores = (rng.integers(0, 300, size=n) / 8192.0).astype(np.float32)
+    assert _select_case(lens, keeps, scores) == 0
+    assert _select_case(lens, keeps, scores, lowest=True, global_idx=True) == 0
+    protect = (rng.random(n) < 0.02).astype(np.uint8)
+    rows = [7, 0, 1, 2, 5, 0]
+    q_idx = np.concatenate([np.sort(rng.choice(max(ln, 1), size=r, replace=False)) for ln, r in zip(lens, rows)])
+    status = _select_case(lens, keeps, scores, protect, rows=rows, q_idx=q_idx, protect_rows=True)
+    assert status & ~fastav.FASTAV_DEV_PROTECT_OVERFLOW == 0
+    smooth = rng.random(n).astype(np.float32)
+    smooth[: longest // 2] = 0.0        # a long run of zeros: equal keys in whole warps
+    assert _select_case(lens, keeps, smooth) == 0
+    assert _select_case(lens, [longest - 1, 0, 0, 33, 1, 999], smooth, global_idx=True) == 0
+
+
 def test_positional_global_prune_keeps_first_audio_tokens():
     """The paper's deployed global stage: a positional rule (here: only the first 10 audio tokens survive,
     everything else is kept) -> keep list -> survivor layout, against the oracle."""
