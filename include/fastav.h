@@ -260,6 +260,57 @@ int32_t fastav_select_noalloc(const fastav_params* params, const float* scores, 
 int32_t fastav_selftest_bounded_wait(int32_t limit_ms, int32_t* device_status, void* stream);
 
 /*
+ * ---- Attention rollout (Section 2.1, "Analysis of audio-visual token importance via attention rollout") ----
+ *
+ * The analysis that tells where the global stage may cut.  For ONE sequence of n tokens and layers 1..L:
+ *
+ *   A^l   [n, n]  head-mean of layer l's attention weights: row i is token i's softmax over the keys it may
+ *                 see (j <= i under FASTAV_CAUSAL), averaged over the Hq query heads (head h reads KV head
+ *                 h / G; softmax scale as in fastav_score)
+ *   Eq. 2         A~^l = alpha A^l + (1 - alpha) I
+ *   Eq. 3         R^l  = A~^l A~^(l-1) ... A~^1
+ *
+ * The running product lives in a caller-owned, opaque STATE buffer (256-byte aligned,
+ * fastav_rollout_state_bytes(n) bytes; the library keeps R transposed, as a pair of bf16 planes whose sum
+ * carries about 16 mantissa bits, twice: one copy is read while the other is written).  Calls, all
+ * asynchronous on `stream`, none allocates:
+ *
+ *   fastav_rollout_begin   R <- I
+ *   fastav_rollout_layer   forms A^l from this layer's q [n, Hq, d] and k [n, Hkv, d] (bf16, strides from
+ *                          params, post-RoPE as the layer's attention uses them), applies Eq. 2 and multiplies
+ *                          it onto R from the left (Eq. 3).  `layer_index` counts the layers applied so far
+ *                          (0 for the first call after begin); it selects which copy of the state is read.
+ *                          lse_opt: NULL, or [n, Hq] fp32 natural-log row sums exp as an attention kernel
+ *                          returns them for this layer (then the statistics pass is skipped).
+ *                          map_out_opt: NULL, or [n, n] fp32 row-major, receives A^l itself (the "raw
+ *                          attention weights" the paper compares the rollout with).
+ *                          Of params: batch (must be 1), total_tokens = total_q = max_seqlen = max_qlen = n,
+ *                          head counts, head_dim (64 or 128), q/k strides, softmax_scale, FASTAV_CAUSAL.
+ *                          Workspace: 256-byte aligned, fastav_rollout_workspace_bytes(params) bytes.
+ *   fastav_rollout_read    importance_out [n] fp32: mean over rows of column j of R, "how much each token
+ *                          from the input layer influences every other token"; rollout_out_opt: NULL or
+ *                          [n, n] fp32 row-major R.  `layers_applied` = number of fastav_rollout_layer calls.
+ *   fastav_rollout_threshold  keep_mask_out [n] uint8 = importance[j] >= threshold, or protect_opt[j] != 0;
+ *                          *cut_out (device int32) = one past the last unprotected token that reaches the
+ *                          threshold (0 if none): the positional rule "drop everything from there on".  The
+ *                          mask feeds fastav_select_mask.
+ *
+ * n <= FASTAV_ROLLOUT_MAX_TOKENS, else FASTAV_ERR_UNSUPPORTED.  Errors as for the other calls; a wait that runs
+ * out inside a kernel sets FASTAV_DEV_WAIT_EXPIRED.  alpha outside [0, 1] is FASTAV_ERR_INVALID_ARG.
+ */
+#define FASTAV_ROLLOUT_MAX_TOKENS 32768
+int32_t fastav_rollout_state_bytes(int32_t n, size_t* out_bytes);
+int32_t fastav_rollout_workspace_bytes(const fastav_params* params, size_t* out_bytes);
+int32_t fastav_rollout_begin(int32_t n, void* state, size_t state_bytes, void* stream);
+int32_t fastav_rollout_layer(const fastav_params* params, const void* q, const void* k, const float* lse_opt, float alpha,
+                             int32_t layer_index, void* state, size_t state_bytes, float* map_out_opt, void* workspace,
+                             size_t workspace_bytes, int32_t* device_status, void* stream);
+int32_t fastav_rollout_read(int32_t n, int32_t layers_applied, const void* state, size_t state_bytes, float* importance_out,
+                            float* rollout_out_opt, void* stream);
+int32_t fastav_rollout_threshold(int32_t n, const float* importance, float threshold, const uint8_t* protect_opt,
+                                 uint8_t* keep_mask_out, int32_t* cut_out, void* stream);
+
+/*
  * Number of kernels this library has launched in this process so far (a diagnostic counter; the
  * only process-wide state the library has).  Benchmarks read it before and after a timed region.
  */

@@ -95,6 +95,9 @@ cudaError_t launch_compact(const Shapes& s, const int32_t* keep_idx, const int32
 // Diagnostic launch counter (fastav_kernel_launches).
 void count_launches(int n);
 
+// The driver's tensor-map encoder (cuTensorMapEncodeTiled), looked up once through the runtime; nullptr if absent.
+void* tensor_map_encode_entry();
+
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // ---- programmatic dependent launch ----------------------------------------------------------------

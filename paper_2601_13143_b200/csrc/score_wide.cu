@@ -94,16 +94,7 @@ __device__ __forceinline__ float2 exp2_pair(float2 x, int pair) {
   return make_float2(ptx::ex2_approx(x.x), ptx::ex2_approx(x.y));
 }
 
-// tcgen05.wait::ld, tied to the registers of the load it completes so that no use can move above it.
-__device__ __forceinline__ void tmem_ld_wait_for(uint32_t (&v)[32]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]), "+r"(v[8]),
-                 "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]), "+r"(v[16]),
-                 "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]), "+r"(v[24]),
-                 "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])
-               :
-               : "memory");
-}
+using ptx::tmem_ld_wait_for;
 
 // Sweep 1, one 32-key piece of a row: fold it into the row's running (max, sum).  Under MASKED,
 // columns above `bound` (relative to the piece's first column) are hidden from this row.  Branch-free:
@@ -753,17 +744,7 @@ using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t
                                    const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult res;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &res) != cudaSuccess ||
-        res != cudaDriverEntryPointSuccess)
-      p = nullptr;
-    return reinterpret_cast<EncodeTiledFn>(p);
-  }();
-  return fn;
-}
+EncodeTiledFn encode_tiled_fn() { return reinterpret_cast<EncodeTiledFn>(tensor_map_encode_entry()); }
 
 // A [rows, heads, d] bf16 tensor with element strides (st, sh, 1) as a rank-3 tensor (d, heads, rows); a box
 // is a 64-element (128-byte) column block of `box_heads` heads of `box_rows` consecutive rows.
@@ -853,6 +834,18 @@ cudaError_t run(const Shapes& s, const Workspace& w, const CUtensorMap& k_map, c
 }
 
 }  // namespace
+
+void* tensor_map_encode_entry() {
+  static void* entry = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult res;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &res) != cudaSuccess ||
+        res != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return p;
+  }();
+  return entry;
+}
 
 // Query rows per block: whole TMA boxes of 8 scored rows x G heads, as many as fit in 256 rows.
 int wide_rows_per_chunk(int group) { return group >= 1 && group <= 32 ? kRowsPerCta / (8 * group) * (8 * group) : 0; }

@@ -37,7 +37,9 @@ FASTAV_ERR_TIMEOUT = -5
 
 EXPORTS = ("fastav_version", "fastav_status_string", "fastav_last_cuda_error", "fastav_workspace_bytes",
            "fastav_score", "fastav_select", "fastav_compact", "fastav_prune", "fastav_host_arena_bytes",
-           "fastav_prune_host", "fastav_kernel_launches", "fastav_select_noalloc", "fastav_select_mask", "fastav_selftest_bounded_wait")
+           "fastav_prune_host", "fastav_kernel_launches", "fastav_select_noalloc", "fastav_select_mask", "fastav_selftest_bounded_wait",
+           "fastav_rollout_state_bytes", "fastav_rollout_workspace_bytes", "fastav_rollout_begin", "fastav_rollout_layer",
+           "fastav_rollout_read", "fastav_rollout_threshold")
 
 
 class fastav_params(ctypes.Structure):
@@ -113,6 +115,20 @@ def library() -> ctypes.CDLL:
         lib.fastav_selftest_bounded_wait.argtypes = [ctypes.c_int32, i32p, vp]
         lib.fastav_select_noalloc.restype = ctypes.c_int32
         lib.fastav_select_noalloc.argtypes = [pp, vp, i32p, i32p, vp, i32p, i32p, i32p, i32p, i32p, vp]
+        szp = ctypes.POINTER(ctypes.c_size_t)
+        lib.fastav_rollout_state_bytes.restype = ctypes.c_int32
+        lib.fastav_rollout_state_bytes.argtypes = [ctypes.c_int32, szp]
+        lib.fastav_rollout_workspace_bytes.restype = ctypes.c_int32
+        lib.fastav_rollout_workspace_bytes.argtypes = [pp, szp]
+        lib.fastav_rollout_begin.restype = ctypes.c_int32
+        lib.fastav_rollout_begin.argtypes = [ctypes.c_int32, vp, ctypes.c_size_t, vp]
+        lib.fastav_rollout_layer.restype = ctypes.c_int32
+        lib.fastav_rollout_layer.argtypes = [pp, vp, vp, vp, ctypes.c_float, ctypes.c_int32, vp, ctypes.c_size_t, vp, vp,
+                                             ctypes.c_size_t, i32p, vp]
+        lib.fastav_rollout_read.restype = ctypes.c_int32
+        lib.fastav_rollout_read.argtypes = [ctypes.c_int32, ctypes.c_int32, vp, ctypes.c_size_t, vp, vp, vp]
+        lib.fastav_rollout_threshold.restype = ctypes.c_int32
+        lib.fastav_rollout_threshold.argtypes = [ctypes.c_int32, vp, ctypes.c_float, vp, vp, i32p, vp]
         _lib = lib
     return _lib
 
@@ -202,6 +218,50 @@ def fastav_select_mask(params, keep_mask, cu_seqlens, keep_idx_out, cu_keep_out,
 def fastav_selftest_bounded_wait(limit_ms: int, device_status, stream=None) -> None:
     """Enqueue the bounded-wait self-test (a wait that cannot succeed; it must end with the error bit set)."""
     _check(library().fastav_selftest_bounded_wait(int(limit_ms), _p(device_status), _stream(stream)), "fastav_selftest_bounded_wait")
+
+
+# ---- attention rollout (Section 2.1, Eq. 2-3): argument marshalling only ------------------------------------
+
+ROLLOUT_MAX_TOKENS = 32768
+
+
+def fastav_rollout_state_bytes(n: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(library().fastav_rollout_state_bytes(int(n), ctypes.byref(out)), "fastav_rollout_state_bytes")
+    return int(out.value)
+
+
+def fastav_rollout_workspace_bytes(params: fastav_params) -> int:
+    out = ctypes.c_size_t(0)
+    _check(library().fastav_rollout_workspace_bytes(ctypes.byref(params), ctypes.byref(out)), "fastav_rollout_workspace_bytes")
+    return int(out.value)
+
+
+def fastav_rollout_begin(n: int, state, stream=None) -> None:
+    """R <- I in the caller's state buffer."""
+    st, st_bytes = _ws(state)
+    _check(library().fastav_rollout_begin(int(n), st, st_bytes, _stream(stream)), "fastav_rollout_begin")
+
+
+def fastav_rollout_layer(params, q, k, alpha: float, layer_index: int, state, workspace, lse_opt=None, map_out_opt=None,
+                         device_status=None, stream=None) -> None:
+    """One layer of Eq. 3: R <- (alpha A^l + (1 - alpha) I) R with A^l the head-mean attention map of (q, k)."""
+    st, st_bytes = _ws(state)
+    ws, ws_bytes = _ws(workspace)
+    _check(library().fastav_rollout_layer(ctypes.byref(params), _p(q), _p(k), _p(lse_opt), float(alpha), int(layer_index), st,
+                                          st_bytes, _p(map_out_opt), ws, ws_bytes, _p(device_status), _stream(stream)),
+           "fastav_rollout_layer")
+
+
+def fastav_rollout_read(n: int, layers_applied: int, state, importance_out, rollout_out_opt=None, stream=None) -> None:
+    st, st_bytes = _ws(state)
+    _check(library().fastav_rollout_read(int(n), int(layers_applied), st, st_bytes, _p(importance_out), _p(rollout_out_opt),
+                                         _stream(stream)), "fastav_rollout_read")
+
+
+def fastav_rollout_threshold(n: int, importance, threshold: float, protect_opt, keep_mask_out, cut_out, stream=None) -> None:
+    _check(library().fastav_rollout_threshold(int(n), _p(importance), float(threshold), _p(protect_opt), _p(keep_mask_out),
+                                              _p(cut_out), _stream(stream)), "fastav_rollout_threshold")
 
 
 NOALLOC_MAX_TOKENS = 1 << 20

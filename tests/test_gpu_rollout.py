@@ -1,0 +1,182 @@
+"""GPU parity of the attention-rollout calls (Section 2.1, Eq. 2-3) against the numpy oracle, through the C ABI.
+
+Tolerances.  The map: fp32 softmax over bf16 inputs, |gpu - ref| <= 2e-3 |ref| + 1e-12 as for the scores (the
+measured error is some 1e-6).  The product: every factor is carried as a pair of bf16 planes (about 16
+mantissa bits) and three of the four partial products are accumulated in fp32, so each layer adds a few
+1e-5 relative; over the paper's 14 layers that stays below 1e-3, which is the bound asserted here.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import rollout as orr
+from conftest import bf16_bits
+from paper_2601_13143_b200 import fastav
+
+pytestmark = pytest.mark.gpu
+
+MAP_RTOL, ROLL_RTOL, ATOL = 2e-3, 1e-3, 1e-12
+
+
+def _layers(seed, n, hq, hkv, d, layers):
+    gen = torch.Generator().manual_seed(seed)
+    return [(torch.randn(n, hq, d, generator=gen).bfloat16(), torch.randn(n, hkv, d, generator=gen).bfloat16()) for _ in range(layers)]
+
+
+def _params(n, hq, hkv, d, q, k, scale, causal):
+    return fastav.make_params(batch=1, total_tokens=n, max_seqlen=n, total_q=n, max_qlen=n, total_keep=0, max_keep=0,
+                              num_q_heads=hq, num_kv_heads=hkv, head_dim=d, hidden=0, q=q, k=k, softmax_scale=scale,
+                              flags=fastav.FASTAV_CAUSAL if causal else 0)
+
+
+def _run(qk, n, hq, hkv, d, scale, causal, alpha, want_maps=False, lse=None):
+    state = torch.empty(fastav.fastav_rollout_state_bytes(n), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    fastav.fastav_rollout_begin(n, state)
+    maps, ws = [], None
+    for l, (q, k) in enumerate(qk):
+        qd, kd = q.cuda(), k.cuda()
+        p = _params(n, hq, hkv, d, qd, kd, scale, causal)
+        if ws is None:
+            ws = torch.empty(fastav.fastav_rollout_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+        m = torch.full((n, n), float("nan"), device="cuda") if want_maps else None
+        fastav.fastav_rollout_layer(p, qd, kd, alpha, l, state, ws, lse_opt=None if lse is None else lse[l].cuda(),
+                                    map_out_opt=m, device_status=status)
+        maps.append(m)
+    imp = torch.full((n,), float("nan"), device="cuda")
+    r = torch.full((n, n), float("nan"), device="cuda")
+    fastav.fastav_rollout_read(n, len(qk), state, imp, r)
+    torch.cuda.synchronize()
+    assert int(status.cpu()) == 0
+    return imp.cpu().double().numpy(), r.cpu().double().numpy(), [None if m is None else m.cpu().double().numpy() for m in maps]
+
+
+def _close(got, ref, rtol, what):
+    assert np.isfinite(got).all(), what
+    err = np.abs(got - ref)
+    bound = rtol * np.abs(ref) + ATOL
+    assert (err <= bound).all(), f"{what}: {(err > bound).sum()} off, worst rel {np.max(err / np.maximum(np.abs(ref), 1e-300)):.3e}"
+    return float(np.max(err / np.maximum(np.abs(ref), 1e-30)))
+
+
+@pytest.mark.parametrize("n,hq,hkv,d", [(300, 8, 2, 64), (333, 28, 4, 128), (128, 4, 4, 128), (1, 2, 1, 64), (129, 6, 3, 64)])
+@pytest.mark.parametrize("causal", [True, False])
+def test_rollout_matches_oracle(n, hq, hkv, d, causal):
+    layers, alpha, scale = 3, 0.5, 1.0 / np.sqrt(d)
+    qk = _layers(n + hq, n, hq, hkv, d, layers)
+    imp, r, maps = _run(qk, n, hq, hkv, d, scale, causal, alpha, want_maps=True)
+    ref_maps = [orr.attention_map(bf16_bits(q), bf16_bits(k), scale, causal) for q, k in qk]
+    for l in range(layers):
+        _close(maps[l], ref_maps[l], MAP_RTOL, f"map of layer {l}")
+        if causal:
+            assert np.array_equal(np.triu(maps[l], 1), np.zeros_like(maps[l]))
+    ref_r = orr.rollout(ref_maps, alpha)
+    _close(r, ref_r, ROLL_RTOL, "rollout")
+    _close(imp, orr.importance(ref_r), ROLL_RTOL, "importance")
+    assert np.allclose(r.sum(axis=1), 1.0, atol=1e-4)
+
+
+def test_rollout_with_the_attention_kernels_lse():
+    """The layer's attention kernel already has log sum exp of every row: handing it in skips the statistics pass."""
+    n, hq, hkv, d, scale, alpha = 257, 8, 4, 128, 0.11, 0.8
+    qk = _layers(5, n, hq, hkv, d, 2)
+    lse = []
+    for q, k in qk:
+        z = torch.einsum("ihd,jhd->ihj", q.double(), k.double().repeat_interleave(hq // hkv, dim=1)) * scale
+        z = z.masked_fill(torch.ones(n, n).triu(1).bool()[:, None, :], float("-inf"))
+        lse.append(torch.logsumexp(z, dim=2).float())
+    imp_a, r_a, _ = _run(qk, n, hq, hkv, d, scale, True, alpha)
+    imp_b, r_b, _ = _run(qk, n, hq, hkv, d, scale, True, alpha, lse=lse)
+    ref = orr.rollout([orr.attention_map(bf16_bits(q), bf16_bits(k), scale, True) for q, k in qk], alpha)
+    _close(r_a, ref, ROLL_RTOL, "own statistics")
+    _close(r_b, ref, ROLL_RTOL, "caller's statistics")
+
+
+def test_rollout_limits_of_eq2():
+    n, hq, hkv, d = 200, 4, 2, 64
+    qk = _layers(9, n, hq, hkv, d, 2)
+    imp, r, _ = _run(qk, n, hq, hkv, d, 0.2, True, 0.0)            # alpha = 0: R = I exactly
+    assert np.array_equal(r, np.eye(n))
+    assert np.allclose(imp, 1.0 / n, rtol=1e-6)
+    imp, r, maps = _run(qk[:1], n, hq, hkv, d, 0.2, True, 1.0, want_maps=True)   # one layer, alpha = 1: R = A
+    _close(r, maps[0], 1e-4, "R = A")
+
+
+def test_rollout_strided_inputs_and_bit_reproducible():
+    n, hq, hkv, d = 260, 8, 2, 64
+    gen = torch.Generator().manual_seed(3)
+    packed = torch.randn(n, hq + 2 * hkv, d, generator=gen).bfloat16()        # q and k as slices of one projection output
+    q, k = packed[:, :hq], packed[:, hq:hq + hkv]
+    imp1, r1, _ = _run([(q, k)], n, hq, hkv, d, 0.125, True, 0.5)
+    imp2, r2, _ = _run([(q.contiguous(), k.contiguous())], n, hq, hkv, d, 0.125, True, 0.5)
+    assert np.array_equal(r1, r2) and np.array_equal(imp1, imp2)
+    ref = orr.rollout([orr.attention_map(bf16_bits(q.contiguous()), bf16_bits(k.contiguous()), 0.125, True)], 0.5)
+    _close(r1, ref, ROLL_RTOL, "strided")
+
+
+def test_threshold_rule_feeds_the_positional_global_stage():
+    """importance -> keep mask and cut position (bit-exact given the fp32 importance) -> keep list."""
+    n, hq, hkv, d = 500, 4, 2, 64
+    imp, _, _ = _run(_layers(11, n, hq, hkv, d, 4), n, hq, hkv, d, 0.125, True, 0.5)
+    imp32 = imp.astype(np.float32)
+    protect = np.zeros(n, dtype=np.uint8)
+    protect[:16] = 1
+    protect[-16:] = 1
+    for threshold, prot in [(float(np.median(imp32)), None), (float(np.quantile(imp32, 0.9)), protect), (2.0, protect), (0.0, None)]:
+        keep = torch.full((n,), 7, dtype=torch.uint8, device="cuda")
+        cut = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+        fastav.fastav_rollout_threshold(n, torch.from_numpy(imp32).cuda(), threshold, None if prot is None else torch.from_numpy(prot).cuda(),
+                                        keep, cut)
+        ref_keep, ref_cut = orr.threshold_rule(imp32, np.float32(threshold), prot)
+        assert keep.cpu().numpy().tolist() == ref_keep.tolist()
+        assert int(cut.cpu()) == ref_cut
+        # the mask is what fastav_select_mask consumes
+        kept = int(ref_keep.sum())
+        p = fastav.make_params(batch=1, total_tokens=n, max_seqlen=n, total_q=0, max_qlen=0, total_keep=max(kept, 1) if kept else 0,
+                               max_keep=kept, num_q_heads=hq, num_kv_heads=hkv, head_dim=d, hidden=0)
+        cu = torch.tensor([0, n], dtype=torch.int32, device="cuda")
+        keep_idx = torch.full((max(kept, 1),), -7, dtype=torch.int32, device="cuda")
+        cu_keep = torch.zeros(2, dtype=torch.int32, device="cuda")
+        ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+        fastav.fastav_select_mask(p, keep, cu, keep_idx, cu_keep, ws)
+        ref_idx, ref_cu = oracle.select_mask(ref_keep, [0, n])
+        assert cu_keep.cpu().tolist() == ref_cu.tolist()
+        assert keep_idx.cpu().numpy()[:kept].tolist() == ref_idx.tolist()
+
+
+def test_rollout_at_the_papers_prompt_size():
+    """About 2,230 tokens, 28 query heads over 4 KV heads of 128 (Section 2.2 and 3.1): four layers against the
+    oracle, then fourteen layers (the middle of a 28-layer model) checked by what must hold at any size."""
+    n, hq, hkv, d, alpha = 2230, 28, 4, 128, 0.5
+    scale = 1.0 / np.sqrt(d)
+    qk = _layers(77, n, hq, hkv, d, 14)
+    imp, r, _ = _run(qk[:4], n, hq, hkv, d, scale, True, alpha)
+    ref = orr.rollout([orr.attention_map(bf16_bits(q), bf16_bits(k), scale, True) for q, k in qk[:4]], alpha)
+    _close(r, ref, ROLL_RTOL, "four layers")
+    _close(imp, orr.importance(ref), ROLL_RTOL, "importance")
+    imp, r, _ = _run(qk, n, hq, hkv, d, scale, True, alpha)
+    assert np.allclose(r.sum(axis=1), 1.0, atol=2e-4)
+    assert np.array_equal(np.triu(r, 1), np.zeros_like(r))
+    assert (r >= 0).all() and abs(imp.sum() - 1.0) < 2e-4
+    assert r[0, 0] == 1.0
+
+
+def test_rollout_argument_errors():
+    n, hq, hkv, d = 64, 4, 2, 64
+    q, k = [t.cuda() for t in _layers(1, n, hq, hkv, d, 1)[0]]
+    p = _params(n, hq, hkv, d, q, k, 0.1, True)
+    state = torch.empty(fastav.fastav_rollout_state_bytes(n), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(fastav.fastav_rollout_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    with pytest.raises(fastav.FastavError):
+        fastav.fastav_rollout_layer(p, q, k, 1.5, 0, state, ws)                   # alpha outside [0, 1]
+    with pytest.raises(fastav.FastavError):
+        fastav.fastav_rollout_layer(p, q, k, 0.5, 0, state[:-256], ws)            # state too small
+    with pytest.raises(fastav.FastavError):
+        fastav.fastav_rollout_layer(p, q, k, 0.5, 0, state, ws[:1024])            # workspace too small
+    p.batch = 2
+    with pytest.raises(fastav.FastavError):
+        fastav.fastav_rollout_layer(p, q, k, 0.5, 0, state, ws)                   # one sequence at a time
+    with pytest.raises(fastav.FastavError):
+        fastav.fastav_rollout_state_bytes(fastav.ROLLOUT_MAX_TOKENS + 1)
+    torch.cuda.synchronize()
