@@ -53,7 +53,8 @@ def measured_peaks():
     if os.path.exists(path):
         with open(path) as f:
             d = json.load(f)
-        return {"hbm_gbs": float(d["hbm_gbs"]), "sm_max_mhz": float(d.get("sm_max_mhz", 1965.0)), "source": "measured"}
+        return {"hbm_gbs": float(d["hbm_gbs"]), "sm_max_mhz": float(d.get("sm_max_mhz", 1965.0)), "source": "measured",
+                "bf16_tflops": d.get("bf16_tflops")}
     return {"hbm_gbs": FALLBACK_HBM_GBS, "sm_max_mhz": 1965.0, "source": "fallback"}
 
 
@@ -272,6 +273,51 @@ def run_oracle_sample(sample) -> None:
                      s["scale"], s["causal"], protect_rows=True)
 
 
+def rollout_line(device, peaks) -> dict:
+    """Secondary measurement: the attention-rollout analysis (Section 2.1, Eq. 2-3) at the paper's prompt size --
+    about 2,230 tokens, a 28-layer model with 28 query heads over 4 KV heads of 128, rolled out to the middle
+    layer (14 layers), causal, alpha = 0.5 -- timed with CUDA events, inputs resident.  Algorithmic work per layer:
+    one causal Q K^T per head (2 d flops per visible pair), one exponential per visible pair and head, and the
+    triangular n x n x n product (n^3 / 3 flops)."""
+    from paper_2601_13143_b200 import fastav
+    n, hq, hkv, d, layers, alpha = 2230, 28, 4, 128, 14, 0.5
+    gen = torch.Generator().manual_seed(2230)
+    qk = [(torch.randn(n, hq, d, generator=gen).bfloat16().to(device), torch.randn(n, hkv, d, generator=gen).bfloat16().to(device))
+          for _ in range(layers)]
+    p = fastav.make_params(batch=1, total_tokens=n, max_seqlen=n, total_q=n, max_qlen=n, total_keep=0, max_keep=0, num_q_heads=hq,
+                           num_kv_heads=hkv, head_dim=d, hidden=0, q=qk[0][0], k=qk[0][1], flags=fastav.FASTAV_CAUSAL)
+    state = torch.empty(fastav.fastav_rollout_state_bytes(n), dtype=torch.uint8, device=device)
+    ws = torch.empty(fastav.fastav_rollout_workspace_bytes(p), dtype=torch.uint8, device=device)
+    imp = torch.empty(n, device=device)
+    status = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def analysis():
+        fastav.fastav_rollout_begin(n, state)
+        for l, (q, k) in enumerate(qk):
+            fastav.fastav_rollout_layer(p, q, k, alpha, l, state, ws, device_status=status)
+        fastav.fastav_rollout_read(n, layers, state, imp)
+
+    for _ in range(3):
+        analysis()
+    torch.cuda.synchronize()
+    reps = 10
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        analysis()
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / reps
+    pairs = n * (n + 1) / 2
+    flops = layers * (hq * pairs * 2 * d + n ** 3 / 3)
+    bf16_peak = peaks.get("bf16_tflops")
+    return {"workload": f"attention rollout, {n} tokens, {hq}/{hkv} heads of {d}, {layers} layers, causal, alpha {alpha}",
+            "ms": round(ms, 4), "ms_per_layer": round(ms / layers, 4), "algorithmic_tflop": round(flops / 1e12, 4),
+            "tflops": round(flops / ms / 1e9, 1), "frac_of_bf16_peak": None if not bf16_peak else round(flops / ms / 1e9 / bf16_peak, 4),
+            "gexp_per_s": round(layers * hq * pairs / ms / 1e6, 1), "importance_sum": round(float(imp.sum()), 6),
+            "device_status": int(status.cpu()), "launches_per_analysis": 2 + 3 * layers}
+
+
 def workload_config(w: W.Workload, lens) -> dict:
     m = w.model
     return {"workload": w.name, "description": w.description, "batch": w.batch, "tokens_per_stage": [sum(x) for x in lens],
@@ -326,6 +372,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-rollout", action="store_true", help="skip the secondary attention-rollout measurement")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -539,6 +586,8 @@ def main():
         cpu = {"value": passes * stoks / dt, "unit": "tokens/s", "cores": oracle.max_threads(), "kind": "oracle", "seconds": round(dt, 3),
                "sample": f"first sequence of each stage ({stoks} tokens) of {w.name}, {passes} passes"}
 
+    rollout = rollout_line(device, peaks) if rank == 0 and world == 1 and not args.no_rollout else None
+
     if rank == 0:
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -549,7 +598,7 @@ def main():
                          "frac_of_nominal_8tbs": round(step_gbs / 8000.0, 4), "of": peaks["source"]},
             "roofline": roofline, "roofline_hbm": roofline_hbm, "compact_roofline": compact_rooflines, "phases": phases,
             "prefill_flops": flops_removed(w, lens), "graph_replay": graph_replay, "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": launches,
-            "device_status": status, "clocks": clocks.summary()}))
+            "device_status": status, "clocks": clocks.summary(), "rollout": rollout}))
     if dist is not None:
         dist.destroy_process_group()
 

@@ -16,8 +16,9 @@
 // the causal mask RT is upper and A~ lower triangular: tiles above the diagonal are written as zeros and the
 // K loop of tile (m, n) only covers the blocks m..n.
 //
-// One CTA per 128 x 128 output tile: warp 0 issues the TMA loads, warp 1 the MMAs, warps 2..9 are the epilogue
-// (thread <-> accumulator row, two warps per 32-lane quarter of TMEM, 64 columns each).  All waits are bounded.
+// One CTA per 128 x 128 output tile: warp 0 issues the TMA loads, warp 1 the MMAs, warps 2..17 are the epilogue
+// (thread <-> accumulator row, four warps per 32-lane quarter of TMEM, 32 columns each: the epilogue, one
+// exponential per element, is what a tile costs, so it gets four warps per scheduler).  All waits are bounded.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <limits.h>
@@ -30,17 +31,18 @@ namespace fastav {
 namespace {
 
 constexpr int kTile = 128;
-constexpr int kThreads = 320;
-constexpr int kEpilogueThreads = 256;
+constexpr int kThreads = 576;
+constexpr int kEpilogueThreads = 512;
+constexpr int kColGroups = 4;  // epilogue warps per TMEM quarter; each takes 32 of the 128 columns
 constexpr int kTmemCols = 256;  // two 128-column accumulators
-constexpr int kMaxStages = 4;
+constexpr int kMaxStages = 6;
 constexpr int kSubTileBytes = kTile * 128;  // 128 rows of one 64-element (128-byte) column block
 
 struct alignas(16) PipeControl {
   uint64_t full[kMaxStages], empty[kMaxStages], tmem_full[2], tmem_empty[2];
   uint32_t tmem_base;
   int abort;
-  float2 part[kTile];  // statistics kernel: (max, sum) of the upper 64 columns, per row
+  float2 part[kColGroups - 1][kTile];  // statistics kernel: (max, sum) per row of column groups 1..3
 };
 
 __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bfloat16& lo) {
@@ -48,10 +50,10 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bflo
   lo = __float2bfloat16_rn(x - __bfloat162float(hi));
 }
 
-// 64 consecutive values of one row as hi / lo planes: 8 stores of 16 bytes each.
-__device__ __forceinline__ void store_split_row(const float (&x)[64], __nv_bfloat16* hi_row, __nv_bfloat16* lo_row) {
+// 32 consecutive values of one row as hi / lo planes: 4 stores of 16 bytes each.
+__device__ __forceinline__ void store_split_row(const float (&x)[32], __nv_bfloat16* hi_row, __nv_bfloat16* lo_row) {
 #pragma unroll
-  for (int c0 = 0; c0 < 64; c0 += 8) {
+  for (int c0 = 0; c0 < 32; c0 += 8) {
     alignas(16) __nv_bfloat16 h[8], l[8];
 #pragma unroll
     for (int c = 0; c < 8; ++c) split_bf16(x[c0 + c], h[c], l[c]);
@@ -103,6 +105,14 @@ __device__ __forceinline__ void drain_loads(PipeControl& ctl, int issued, int st
 }
 
 // ---- the attention map ---------------------------------------------------------------------------
+template <int DIM, int MODE>
+struct AttnSmem {
+  static constexpr int kOperandBytes = (DIM / 64) * kSubTileBytes;
+  static constexpr int kSlots = MODE == 0 ? 1 : 3;
+  static constexpr int kStages = 6 - kSlots;  // six tiles in all: 192 KB at head_dim 128
+  static constexpr size_t kBytes = (size_t)6 * kOperandBytes + sizeof(PipeControl) + 1024;
+};
+
 // MODE 0: grid (row blocks, heads); the block walks the key blocks its rows may see and leaves, per row, the
 //         log2-sum-exp2 of the scaled logits of head blockIdx.y in lse2_out[head][row].
 // MODE 1: grid (row blocks, key blocks); the block walks the heads and accumulates the softmax weights of its
@@ -114,17 +124,24 @@ rollout_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
                     const float* __restrict__ lse, long long lse_row, long long lse_head, float lse_mult, float alpha,
                     __nv_bfloat16* __restrict__ a_hi, __nv_bfloat16* __restrict__ a_lo, float* __restrict__ map_out,
                     int32_t* device_status) {
-  constexpr int kStages = DIM == 128 ? 3 : 4;
+  // Shared memory: a ring of tiles of the operand that changes every iteration (MODE 0: the K tile of the key
+  // block; MODE 1: the Q tile of the head) and a few slots for the one that changes rarely (MODE 0: the Q tile,
+  // loaded once; MODE 1: the K tile, loaded once per KV head and shared by the G heads of its group -- three
+  // slots used in turn, so that a slot is overwritten no sooner than three iterations after its last use,
+  // which is the distance the ring's own barriers already guarantee).
+  using Cfg = AttnSmem<DIM, MODE>;
+  constexpr int kStages = Cfg::kStages, kSlots = Cfg::kSlots;
   constexpr int kSubTiles = DIM / 64;
-  constexpr int kOperandBytes = kSubTiles * kSubTileBytes;  // one 128 x DIM tile
-  constexpr int kStageBytes = 2 * kOperandBytes;            // the Q tile, then the K tile
+  constexpr int kOperandBytes = Cfg::kOperandBytes;  // one 128 x DIM tile
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
-  PipeControl& ctl = *reinterpret_cast<PipeControl*>(smem_raw + (base - ptx::smem_u32(smem_raw)) + kStages * kStageBytes);
+  const uint32_t slots = base + kStages * kOperandBytes;
+  PipeControl& ctl = *reinterpret_cast<PipeControl*>(smem_raw + (base - ptx::smem_u32(smem_raw)) + (kStages + kSlots) * kOperandBytes);
   volatile int* abort = &ctl.abort;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int rb = blockIdx.x;
   const int blocks = n_pad / kTile;
+  // Under the causal mask the last row block has the most key blocks to walk: the statistics kernel starts those first.
+  const int rb = (MODE == 0 && causal) ? blocks - 1 - (int)blockIdx.x : (int)blockIdx.x;
 
   if (MODE == 1 && causal && (int)blockIdx.y > rb) {
     // a tile no row may see: zeros (uniform for the block, before anything is set up)
@@ -154,12 +171,15 @@ rollout_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
         if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.empty[stage]), ((it / kStages) & 1) ^ 1u, abort)) break;
         const int head = MODE == 0 ? (int)blockIdx.y : it, jb = MODE == 0 ? it : (int)blockIdx.y;
         const uint32_t bar = ptx::smem_u32(&ctl.full[stage]);
-        const uint32_t q_dst = base + stage * kStageBytes, k_dst = q_dst + kOperandBytes;
-        ptx::mbar_arrive_expect_tx(bar, kStageBytes);
+        const bool load_q = MODE == 1 || it == 0, load_k = MODE == 0 || it % group == 0;
+        const uint32_t ring = base + stage * kOperandBytes;
+        const uint32_t q_dst = MODE == 0 ? slots : ring;
+        const uint32_t k_dst = MODE == 0 ? ring : slots + ((it / group) % kSlots) * kOperandBytes;
+        ptx::mbar_arrive_expect_tx(bar, (load_q ? kOperandBytes : 0) + (load_k ? kOperandBytes : 0));
 #pragma unroll
         for (int sub = 0; sub < kSubTiles; ++sub) {
-          ptx::tma_load_3d(q_dst + sub * kSubTileBytes, &q_map, sub * 64, head, rb * kTile, bar);
-          ptx::tma_load_3d(k_dst + sub * kSubTileBytes, &k_map, sub * 64, head / group, jb * kTile, bar);
+          if (load_q) ptx::tma_load_3d(q_dst + sub * kSubTileBytes, &q_map, sub * 64, head, rb * kTile, bar);
+          if (load_k) ptx::tma_load_3d(k_dst + sub * kSubTileBytes, &k_map, sub * 64, head / group, jb * kTile, bar);
         }
       }
       if (*abort) drain_loads(ctl, it, kStages);
@@ -171,7 +191,9 @@ rollout_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
         if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.full[stage]), (it / kStages) & 1, abort)) break;
         if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.tmem_empty[buf]), ((it >> 1) & 1) ^ 1u, abort)) break;
         ptx::tc_fence_after_sync();
-        const uint32_t q_tile = base + stage * kStageBytes, k_tile = q_tile + kOperandBytes;
+        const uint32_t ring = base + stage * kOperandBytes;
+        const uint32_t q_tile = MODE == 0 ? slots : ring;
+        const uint32_t k_tile = MODE == 0 ? ring : slots + ((it / group) % kSlots) * kOperandBytes;
 #pragma unroll
         for (int ks = 0; ks < DIM / 16; ++ks) {
           const uint32_t sub = ks / 4, off = (ks % 4) * 32;
@@ -183,75 +205,92 @@ rollout_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
       }
     }
   } else {
-    const int quarter = warp & 3, half = (warp - 2) >> 2;  // TMEM lanes 32 quarter .., columns 64 half ..
+    const int quarter = warp & 3, cg = (warp - 2) >> 2;  // TMEM lanes 32 quarter .., columns 32 cg ..
     const int row_in = quarter * 32 + lane, row = rb * kTile + row_in;
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
     const int last_visible = min(n - 1, causal ? row : INT_MAX);
     float zmax = -INFINITY, sum = 0.f;  // MODE 0, in scaled log2 units
-    float acc[64];                      // MODE 1
+    float acc[32];                      // MODE 1
 #pragma unroll
-    for (int c = 0; c < 64; ++c) acc[c] = 0.f;
+    for (int c = 0; c < 32; ++c) acc[c] = 0.f;
     bool ok = true;
+    // MODE 1: the row's statistic of the NEXT head is fetched while this head's tile is worked on
+    float lse_next = (MODE == 1 && row < n) ? lse[row * lse_row] : 0.f;
     for (int it = 0; it < iters; ++it) {
       const int buf = it & 1;
+      const float lse_here = lse_next;
+      if (MODE == 1 && row < n && it + 1 < iters) lse_next = lse[row * lse_row + (it + 1) * lse_head];
       ok = ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.tmem_full[buf]), (it >> 1) & 1, abort);
       if (!ok) break;
       ptx::tc_fence_after_sync();
-      const int head = MODE == 0 ? (int)blockIdx.y : it, jb = MODE == 0 ? it : (int)blockIdx.y;
-      uint32_t va[32], vb[32];
-      const uint32_t taddr = lane_addr + buf * kTile + half * 64;
-      ptx::tmem_ld32(taddr, va);
-      ptx::tmem_ld32(taddr + 32, vb);
-      ptx::tmem_ld_wait_for(va);
-      ptx::tmem_ld_wait_for(vb);
+      const int jb = MODE == 0 ? it : (int)blockIdx.y;
+      uint32_t v[32];
+      ptx::tmem_ld32(lane_addr + buf * kTile + cg * 32, v);
+      ptx::tmem_ld_wait_for(v);
       ptx::tc_fence_before_sync();
       ptx::mbar_arrive(ptx::smem_u32(&ctl.tmem_empty[buf]));  // the accumulator may be overwritten
-      const int limit = last_visible - (jb * kTile + half * 64);  // columns 0..limit of this half are visible
+      const int limit = last_visible - (jb * kTile + cg * 32);  // columns 0..limit of this group are visible
+      if (limit < 0) continue;
+      const bool whole = limit >= 31;  // the usual case; only tiles on the diagonal or at the end of the sequence are cut
       if constexpr (MODE == 0) {
         float tile_max = -INFINITY;
+        if (whole) {
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          if (c <= limit) tile_max = fmaxf(tile_max, __uint_as_float(va[c]));
-          if (c + 32 <= limit) tile_max = fmaxf(tile_max, __uint_as_float(vb[c]));
+          for (int c = 0; c < 32; ++c) tile_max = fmaxf(tile_max, __uint_as_float(v[c]));
+        } else {
+#pragma unroll
+          for (int c = 0; c < 32; ++c)
+            if (c <= limit) tile_max = fmaxf(tile_max, __uint_as_float(v[c]));
         }
-        if (tile_max > -INFINITY) {
-          const float new_max = fmaxf(zmax, tile_max * scale_log2);
-          float add = 0.f;
+        const float new_max = fmaxf(zmax, tile_max * scale_log2);
+        float add0 = 0.f, add1 = 0.f;
+        if (whole) {
 #pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            if (c <= limit) add += ptx::ex2_approx(__uint_as_float(va[c]) * scale_log2 - new_max);
-            if (c + 32 <= limit) add += ptx::ex2_approx(__uint_as_float(vb[c]) * scale_log2 - new_max);
+          for (int c = 0; c < 32; c += 2) {
+            add0 += ptx::ex2_approx(fmaf(__uint_as_float(v[c]), scale_log2, -new_max));
+            add1 += ptx::ex2_approx(fmaf(__uint_as_float(v[c + 1]), scale_log2, -new_max));
           }
-          sum = sum * ptx::ex2_approx(zmax - new_max) + add;  // zmax = -inf the first time: the factor is 0
-          zmax = new_max;
-        }
-      } else {
-        const float neg_lse2 = row < n ? -lse[row * lse_row + head * lse_head] * lse_mult : 0.f;
+        } else {
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          if (c <= limit) acc[c] += ptx::ex2_approx(fmaf(__uint_as_float(va[c]), scale_log2, neg_lse2));
-          if (c + 32 <= limit) acc[c + 32] += ptx::ex2_approx(fmaf(__uint_as_float(vb[c]), scale_log2, neg_lse2));
+          for (int c = 0; c < 32; ++c)
+            if (c <= limit) add0 += ptx::ex2_approx(fmaf(__uint_as_float(v[c]), scale_log2, -new_max));
+        }
+        sum = sum * ptx::ex2_approx(zmax - new_max) + (add0 + add1);  // zmax = -inf the first time: the factor is 0
+        zmax = new_max;
+      } else {
+        const float neg_lse2 = -lse_here * lse_mult;
+        if (whole) {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) acc[c] += ptx::ex2_approx(fmaf(__uint_as_float(v[c]), scale_log2, neg_lse2));
+        } else {
+#pragma unroll
+          for (int c = 0; c < 32; ++c)
+            if (c <= limit) acc[c] += ptx::ex2_approx(fmaf(__uint_as_float(v[c]), scale_log2, neg_lse2));
         }
       }
     }
     if constexpr (MODE == 0) {
-      // the two halves of a row meet in shared memory; the lower half writes the result
-      if (half == 1) ctl.part[row_in] = make_float2(zmax, sum);
+      // the four column groups of a row meet in shared memory; group 0 writes the result
+      if (cg > 0) ctl.part[cg - 1][row_in] = make_float2(zmax, sum);
       asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory");
-      if (half == 0 && ok && !*abort) {
-        const float2 other = ctl.part[row_in];
-        const float m = fmaxf(zmax, other.x);
-        float total = 0.f;
-        if (zmax > -INFINITY) total += sum * ptx::ex2_approx(zmax - m);
-        if (other.x > -INFINITY) total += other.y * ptx::ex2_approx(other.x - m);
+      if (cg == 0 && ok && !*abort) {
+        float m = zmax;
+#pragma unroll
+        for (int g = 0; g < kColGroups - 1; ++g) m = fmaxf(m, ctl.part[g][row_in].x);
+        float total = zmax > -INFINITY ? sum * ptx::ex2_approx(zmax - m) : 0.f;
+#pragma unroll
+        for (int g = 0; g < kColGroups - 1; ++g) {
+          const float2 other = ctl.part[g][row_in];
+          if (other.x > -INFINITY) total += other.y * ptx::ex2_approx(other.x - m);
+        }
         lse2_out[(long long)blockIdx.y * n_pad + row] = total > 0.f ? m + log2f(total) : INFINITY;  // a row that sees nothing adds 0
       }
     } else if (ok) {
-      const int col0 = blockIdx.y * kTile + half * 64;
+      const int col0 = blockIdx.y * kTile + cg * 32;
       const float inv_heads = 1.0f / (float)hq;
-      float x[64];
+      float x[32];
 #pragma unroll
-      for (int c = 0; c < 64; ++c) {
+      for (int c = 0; c < 32; ++c) {
         const float a = row < n ? acc[c] * inv_heads : 0.f;
         if (map_out && row < n && col0 + c < n) map_out[(long long)row * n + col0 + c] = a;
         x[c] = alpha * a + ((row < n && col0 + c == row) ? 1.0f - alpha : 0.f);  // Eq. 2
@@ -264,20 +303,33 @@ rollout_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
 }
 
 // ---- Eq. 3: RT_new = RT_old * A~^T ------------------------------------------------------------------
-// Grid (n_pad / 128, n_pad / 128): block (m, nn) computes RT_new[128 m .., 128 nn ..].  K runs three times
-// over the needed 64-wide blocks: (RT hi, A~ hi), (RT lo, A~ hi), (RT hi, A~ lo).
+// Grid (n_pad / 128, n_pad / 128): one block per 128 x 128 tile of RT_new.  Per 64-wide K block the four
+// operand tiles (RT hi, RT lo, A~ hi, A~ lo) are loaded once and used for the three products
+// RT hi * A~ hi, RT lo * A~ hi, RT hi * A~ lo, all accumulated into the same TMEM tile.
 __global__ void __launch_bounds__(kThreads, 1)
 rollout_gemm_kernel(const __grid_constant__ CUtensorMap rt_hi_map, const __grid_constant__ CUtensorMap rt_lo_map,
                     const __grid_constant__ CUtensorMap a_hi_map, const __grid_constant__ CUtensorMap a_lo_map, int n_pad,
                     int causal, __nv_bfloat16* __restrict__ out_hi, __nv_bfloat16* __restrict__ out_lo, int32_t* device_status) {
-  constexpr int kStages = 4;
-  constexpr int kStageBytes = 2 * kSubTileBytes;  // 128 x 64 of RT, then 128 x 64 of A~
+  constexpr int kStages = 3;
+  constexpr int kStageBytes = 4 * kSubTileBytes;  // 128 x 64 each of RT hi, RT lo, A~ hi, A~ lo
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   PipeControl& ctl = *reinterpret_cast<PipeControl*>(smem_raw + (base - ptx::smem_u32(smem_raw)) + kStages * kStageBytes);
   volatile int* abort = &ctl.abort;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int mb = blockIdx.x, nb = blockIdx.y;
+  // Tile of this block.  Under the causal mask tile (m, nn) has a K loop of nn - m + 1 blocks: the blocks are handed
+  // out by decreasing nn - m (longest first, so that the short ones fill the tail), the all-zero tiles last.
+  int mb = blockIdx.x, nb = blockIdx.y;
+  if (causal) {
+    const int blocks = gridDim.x;
+    int id = blockIdx.y * blocks + blockIdx.x, diag = blocks - 1;  // diag = nn - m, from blocks - 1 down to -(blocks - 1)
+    while (id >= blocks - abs(diag)) {
+      id -= blocks - abs(diag);
+      --diag;
+    }
+    mb = diag >= 0 ? id : id - diag;
+    nb = mb + diag;
+  }
 
   if (causal && mb > nb) {  // RT is upper triangular: nothing but zeros here
     for (int i = threadIdx.x; i < kTile * (kTile / 8); i += kThreads) {
@@ -290,7 +342,7 @@ rollout_gemm_kernel(const __grid_constant__ CUtensorMap rt_hi_map, const __grid_
   }
   // 64-wide K blocks: RT[m][k] is zero for k < m, A~[nn][k] for k > nn
   const int kb_lo = causal ? mb * 2 : 0, kb_hi = causal ? (nb + 1) * 2 : n_pad / 64;
-  const int per_pass = kb_hi - kb_lo, iters = 3 * per_pass;
+  const int iters = kb_hi - kb_lo;
 
   pipe_setup(ctl, kStages, warp, &rt_hi_map, &a_hi_map);
   const uint32_t tmem = ctl.tmem_base;
@@ -301,12 +353,14 @@ rollout_gemm_kernel(const __grid_constant__ CUtensorMap rt_hi_map, const __grid_
       for (; it < iters; ++it) {
         const int stage = it % kStages;
         if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.empty[stage]), ((it / kStages) & 1) ^ 1u, abort)) break;
-        const int pass = it / per_pass, kb = kb_lo + it % per_pass;
+        const int kb = kb_lo + it;
         const uint32_t bar = ptx::smem_u32(&ctl.full[stage]);
-        const uint32_t rt_dst = base + stage * kStageBytes, a_dst = rt_dst + kSubTileBytes;
+        const uint32_t dst = base + stage * kStageBytes;
         ptx::mbar_arrive_expect_tx(bar, kStageBytes);
-        ptx::tma_load_2d(rt_dst, pass == 1 ? &rt_lo_map : &rt_hi_map, kb * 64, mb * kTile, bar);
-        ptx::tma_load_2d(a_dst, pass == 2 ? &a_lo_map : &a_hi_map, kb * 64, nb * kTile, bar);
+        ptx::tma_load_2d(dst, &rt_hi_map, kb * 64, mb * kTile, bar);
+        ptx::tma_load_2d(dst + kSubTileBytes, &rt_lo_map, kb * 64, mb * kTile, bar);
+        ptx::tma_load_2d(dst + 2 * kSubTileBytes, &a_hi_map, kb * 64, nb * kTile, bar);
+        ptx::tma_load_2d(dst + 3 * kSubTileBytes, &a_lo_map, kb * 64, nb * kTile, bar);
       }
       if (*abort) drain_loads(ctl, it, kStages);
     }
@@ -318,33 +372,32 @@ rollout_gemm_kernel(const __grid_constant__ CUtensorMap rt_hi_map, const __grid_
         ok = ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.full[stage]), (it / kStages) & 1, abort);
         if (!ok) break;
         ptx::tc_fence_after_sync();
-        const uint32_t rt_tile = base + stage * kStageBytes, a_tile = rt_tile + kSubTileBytes;
+        const uint32_t rt_hi = base + stage * kStageBytes, rt_lo = rt_hi + kSubTileBytes, a_hi = rt_hi + 2 * kSubTileBytes,
+                       a_lo = rt_hi + 3 * kSubTileBytes;
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
-          ptx::umma_bf16(tmem, ptx::umma_desc_sw128(rt_tile, ks * 32), ptx::umma_desc_sw128(a_tile, ks * 32),
-                         ptx::umma_idesc_bf16(kTile, kTile), (it > 0 || ks > 0) ? 1u : 0u);
+        for (int term = 0; term < 3; ++term) {
+          const uint32_t rt_tile = term == 1 ? rt_lo : rt_hi, a_tile = term == 2 ? a_lo : a_hi;
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)
+            ptx::umma_bf16(tmem, ptx::umma_desc_sw128(rt_tile, ks * 32), ptx::umma_desc_sw128(a_tile, ks * 32),
+                           ptx::umma_idesc_bf16(kTile, kTile), (it > 0 || term > 0 || ks > 0) ? 1u : 0u);
+        }
         ptx::umma_commit(ptx::smem_u32(&ctl.empty[stage]));
       }
       if (ok) ptx::umma_commit(ptx::smem_u32(&ctl.tmem_full[0]));
     }
   } else {
-    const int quarter = warp & 3, half = (warp - 2) >> 2;
+    const int quarter = warp & 3, cg = (warp - 2) >> 2;
     const int row = mb * kTile + quarter * 32 + lane;
     if (ptx::mbar_wait_bounded(ptx::smem_u32(&ctl.tmem_full[0]), 0, abort)) {
       ptx::tc_fence_after_sync();
-      uint32_t va[32], vb[32];
-      const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + half * 64;
-      ptx::tmem_ld32(taddr, va);
-      ptx::tmem_ld32(taddr + 32, vb);
-      ptx::tmem_ld_wait_for(va);
-      ptx::tmem_ld_wait_for(vb);
-      float x[64];
+      uint32_t v[32];
+      ptx::tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + cg * 32, v);
+      ptx::tmem_ld_wait_for(v);
+      float x[32];
 #pragma unroll
-      for (int c = 0; c < 32; ++c) {
-        x[c] = __uint_as_float(va[c]);
-        x[c + 32] = __uint_as_float(vb[c]);
-      }
-      const long long at = (long long)row * n_pad + nb * kTile + half * 64;
+      for (int c = 0; c < 32; ++c) x[c] = __uint_as_float(v[c]);
+      const long long at = (long long)row * n_pad + nb * kTile + cg * 32;
       store_split_row(x, out_hi + at, out_lo + at);
     }
   }
@@ -459,8 +512,8 @@ template <int DIM>
 cudaError_t run_layer(const fastav_params& p, const CUtensorMap& q_map, const CUtensorMap& k_map, const float* lse_opt,
                       float alpha, float* lse2, __nv_bfloat16* a_hi, __nv_bfloat16* a_lo, float* map_out,
                       int32_t* device_status, cudaStream_t stream) {
-  constexpr int kStages = DIM == 128 ? 3 : 4;
-  constexpr size_t smem = (size_t)kStages * 2 * (DIM / 64) * kSubTileBytes + sizeof(PipeControl) + 1024;
+  constexpr size_t smem = AttnSmem<DIM, 0>::kBytes;
+  static_assert(AttnSmem<DIM, 0>::kBytes == AttnSmem<DIM, 1>::kBytes, "both kernels are launched with the same size");
   const int n = p.total_tokens, n_pad = pad_of(n), blocks = n_pad / kTile;
   const int causal = (p.flags & FASTAV_CAUSAL) ? 1 : 0;
   const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
@@ -559,7 +612,7 @@ extern "C" int32_t fastav_rollout_layer(const fastav_params* p, const void* q, c
                       ? run_layer<128>(*p, q_map, k_map, lse_opt, alpha, lse2, a_hi, a_lo, map_out_opt, device_status, st)
                       : run_layer<64>(*p, q_map, k_map, lse_opt, alpha, lse2, a_hi, a_lo, map_out_opt, device_status, st);
   if (e != cudaSuccess) return FASTAV_ERR_CUDA;
-  constexpr size_t gemm_smem = 4 * 2 * kSubTileBytes + sizeof(PipeControl) + 1024;
+  constexpr size_t gemm_smem = 3 * 4 * kSubTileBytes + sizeof(PipeControl) + 1024;
   e = cudaFuncSetAttribute(rollout_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem);
   if (e != cudaSuccess) return FASTAV_ERR_CUDA;
   rollout_gemm_kernel<<<dim3(n_pad / kTile, n_pad / kTile), kThreads, gemm_smem, st>>>(
