@@ -363,6 +363,46 @@ def test_compact_matches_oracle(hkv, d, hid, path):
     parity.assert_bits_equal(buf.k_out, ref["k"], "k (global indices)")
 
 
+@pytest.mark.parametrize("path", [0, fastav.FASTAV_COMPACT_PATH_LOADSTORE])
+def test_compact_buffers_beyond_4_gib(path):
+    """Byte offsets past 2^32: 1.2 M tokens of 2,048 bf16 hidden values (4.9 GB in, 1.6 GB out), three sequences,
+    every third token kept through a rule-given mask.  Expected rows by plain indexing on the same tensors."""
+    n_seq, per_seq, hid, hkv, d = 3, 400_000, 2048, 1, 64
+    n = n_seq * per_seq
+    dev = "cuda"
+    rows = torch.arange(n, device=dev, dtype=torch.int32)
+    hidden = torch.empty(n, hid, dtype=torch.bfloat16, device=dev)
+    cols = (torch.arange(hid, device=dev, dtype=torch.int32) % 7).view(1, hid)
+    for i in range(0, n, 100_000):                       # row id and column pattern in every element, built in slices
+        hidden[i:i + 100_000] = ((rows[i:i + 100_000].view(-1, 1) % 251) + cols).to(torch.bfloat16)
+    k = (rows % 509).view(n, 1, 1).expand(n, hkv, d).to(torch.bfloat16).contiguous()
+    pos = rows.clone()
+    mask = (rows % 3 == 1).to(torch.uint8)
+    kept = int(mask.sum())
+    cu = torch.tensor([0, per_seq, 2 * per_seq, n], dtype=torch.int32, device=dev)
+    p = fastav.make_params(batch=n_seq, total_tokens=n, max_seqlen=per_seq, total_q=0, max_qlen=0, total_keep=kept,
+                           max_keep=kept, num_q_heads=hkv, num_kv_heads=hkv, head_dim=d, hidden=hid, k=k, flags=path)
+    keep_idx = torch.empty(kept, dtype=torch.int32, device=dev)
+    cu_keep = torch.empty(n_seq + 1, dtype=torch.int32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws = torch.empty(max(fastav.fastav_workspace_bytes(p), 256), dtype=torch.uint8, device=dev)
+    fastav.fastav_select_mask(p, mask, cu, keep_idx, cu_keep, ws, status)
+    hidden_out = torch.empty(kept, hid, dtype=torch.bfloat16, device=dev)
+    k_out = torch.empty(kept, hkv, d, dtype=torch.bfloat16, device=dev)
+    pos_out = torch.empty(kept, dtype=torch.int32, device=dev)
+    fastav.fastav_compact(p, keep_idx, cu_keep, cu, hidden_in=hidden, hidden_out=hidden_out, pos_in=pos, pos_out=pos_out,
+                          k_in=k, k_out=k_out, device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.cpu()) == 0
+    src = torch.nonzero(mask).view(-1)                   # survivors in order, as global row numbers
+    assert torch.equal(pos_out.long(), src)
+    assert cu_keep.cpu().tolist() == [0] + torch.cumsum(mask.view(n_seq, per_seq).sum(dim=1), 0).tolist()
+    for i in range(0, kept, 50_000):
+        idx = src[i:i + 50_000]
+        assert torch.equal(hidden_out[i:i + 50_000].view(torch.int16), hidden[idx].view(torch.int16)), f"hidden rows from {i}"
+        assert torch.equal(k_out[i:i + 50_000].view(torch.int16), k[idx].view(torch.int16)), f"k rows from {i}"
+
+
 def test_compact_many_rows_per_warp_and_bad_rows_in_between():
     """Enough rows that every warp of the bulk-copy kernel cycles its slots many times, with a few
     out-of-range indices sprinkled in (skipped rows must not disturb the rows around them)."""
