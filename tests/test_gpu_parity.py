@@ -494,6 +494,41 @@ def test_prune_small_problems(lens, rows, keeps, hq, hkv, d, hid, protect_rows):
                            getattr(buf, k).view(torch.int32) if t.dtype == torch.float32 else getattr(buf, k).view(torch.int16) if t.dtype == torch.bfloat16 else getattr(buf, k)), k
 
 
+@pytest.mark.parametrize("seed", range(120))
+def test_prune_random_shapes(seed):
+    """Seeded random problems: batch, ragged lengths (empty ones too), scored rows anywhere in the sequence or
+    trailing, head counts, head size, keep counts from 0 to n, duplicate keys (exact ties), a protect mask, the
+    causal flag and the score path all drawn at random; the whole fused call against the oracle."""
+    rng = np.random.default_rng(1000 + seed)
+    batch = int(rng.integers(1, 7))
+    lens = [int(rng.choice([0, 1, 2, 31, 64, 127, 128, 129, 300, 515, 1025, 2049])) if rng.random() < 0.5 else int(rng.integers(1, 900))
+            for _ in range(batch)]
+    if sum(lens) == 0:
+        lens[0] = 5
+    max_rows = int(rng.choice([1, 2, 4, 5, 17, 64, 130]))
+    rows = [int(rng.integers(0, max_rows + 1)) for _ in lens]
+    hkv = int(rng.choice([1, 2, 4]))
+    hq = hkv * int(rng.choice([1, 2, 4, 7]))
+    d = int(rng.choice([64, 128]))
+    keeps = [int(rng.integers(0, n + 1)) for n in lens]
+    p = W.random_problem(seed=seed, lens=lens, rows=rows, keeps=keeps, num_q_heads=hq, num_kv_heads=hkv, head_dim=d,
+                         hidden=int(rng.choice([64, 136, 512])), duplicate_keys=int(rng.integers(0, 5)),
+                         trailing_rows=bool(rng.random() < 0.5))
+    p.causal = bool(rng.random() < 0.7)
+    p.protect_rows = bool(rng.random() < 0.5)
+    p.softmax_scale = float(rng.choice([1.0 / np.sqrt(d), 0.05, 0.3]))
+    protect = (torch.from_numpy(rng.random(sum(lens))) < 0.04).to(torch.uint8) if rng.random() < 0.5 else None
+    path = str(rng.choice(["auto", "auto", "generic", "narrow", "wide"]))
+    if not _path_applies(path, [min(r, n) for r, n in zip(rows, lens)], hq, hkv, d):
+        path = "auto"
+    buf = parity.to_device(p, protect=protect, extra_flags=SCORE_PATHS[path])
+    buf.prune()
+    torch.cuda.synchronize()
+    ref = parity.oracle_prune(p, protect=protect)
+    stats = parity.check_fused_against_oracle(p, buf, ref, protect=protect, what=f"seed {seed}: lens={lens} rows={rows} hq={hq} hkv={hkv} d={d} {path}")
+    assert stats["device_status"] & ~fastav.FASTAV_DEV_PROTECT_OVERFLOW == 0
+
+
 def test_prune_with_protect_mask_keeps_all_text_tokens():
     w = W.WORKLOADS["c1_tiny"]
     p = W.make_stage(w, 0)
