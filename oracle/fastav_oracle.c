@@ -12,7 +12,7 @@
  *
  * What it computes (paper, Section 2.2, "Fine pruning", Eq. 4):
  *     s = mean_h softmax(Q_last K^T)
- * generalised the way the build's scope states it: R scored query rows instead
+ * generalised to R scored query rows instead
  * of one (mean over rows and heads), grouped-query attention (query head h
  * reads KV head h / G), an optional causal mask by token index, an explicit
  * softmax scale, and variable-length batches.  Then "tokens with the lowest P%

@@ -1,7 +1,7 @@
 """Shared helpers of the GPU parity tests: move a generated problem to the device, run the oracle
 on the same bits, and compare under the stated rules.
 
-Rules (from the build's target statement):
+Rules:
   scores      |gpu - ref| <= 2e-3 |ref| + 1e-12      (fp32 accumulation over bf16 inputs)
   keep sets   identical to the oracle's, except tokens whose oracle score lies within 2e-3 relative of
               the oracle's k-th score ("ambiguous"); those are counted and returned
