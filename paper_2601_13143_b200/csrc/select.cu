@@ -108,15 +108,17 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
       // log2-sum-exp2 of one row of logits by one warp: running (max, sum) per lane, merged in a fixed order
       const float* z = fl.logits + ((long long)(i / rows) * fl.rq + i % rows) * s.total_tokens + tok0;
       float m = -INFINITY, l = 0.f;
-      for (int j0 = lane; j0 < n; j0 += 128) {
-        float v[4];
+      for (int j0 = lane; j0 < n; j0 += 512) {  // sixteen loads in flight per lane: at most two trips for 1,024 tokens
+        float v[16];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) v[u] = j0 + 32 * u < n ? z[j0 + 32 * u] : -INFINITY;
-        const float m_new = fmaxf(fmaxf(m, fmaxf(v[0], v[1])), fmaxf(v[2], v[3]));
+        for (int u = 0; u < 16; ++u) v[u] = j0 + 32 * u < n ? z[j0 + 32 * u] : -INFINITY;
+        float m_new = m;
+#pragma unroll
+        for (int u = 0; u < 16; ++u) m_new = fmaxf(m_new, v[u]);
         if (m_new > -INFINITY) {
           l = l * exp2f(m - m_new);
 #pragma unroll
-          for (int u = 0; u < 4; ++u) l += exp2f(v[u] - m_new);
+          for (int u = 0; u < 16; ++u) l += exp2f(v[u] - m_new);
           m = m_new;
         }
       }
@@ -132,15 +134,15 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
     for (int j = tid; j < n; j += kThreads) {
       const float* z = fl.logits + tok0 + j;
       float total = 0.f;
-      for (int i0 = 0; i0 < terms; i0 += 8) {
-        float v[8];
+      for (int i0 = 0; i0 < terms; i0 += 16) {
+        float v[16];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < 16; ++u) {
           const int i = i0 + u;
           v[u] = i < terms ? z[((long long)(i / rows) * fl.rq + i % rows) * s.total_tokens] : -INFINITY;
         }
 #pragma unroll
-        for (int u = 0; u < 8; ++u)
+        for (int u = 0; u < 16; ++u)
           if (i0 + u < terms) total += exp2f(v[u] - lse_sh[i0 + u]);
       }
       const float score = all_rows > 0 ? total / ((float)s.hq * (float)all_rows) : 0.f;
