@@ -104,6 +104,9 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
     float* lse_sh = reinterpret_cast<float*>(keys + (s.max_seqlen + s.max_seqlen / 32 + 1));
     const int row0 = cu_qlens[b], all_rows = cu_qlens[b + 1] - row0, rows = min(all_rows, fl.rq);
     const int terms = s.hq * rows;  // term i = (head i / rows, row i % rows)
+    // where term i's logits start, in units of N floats: worked out once, not per token (no integer division in the loop below)
+    int* term_row = reinterpret_cast<int*>(lse_sh + s.hq * fl.rq);
+    for (int i = tid; i < terms; i += kThreads) term_row[i] = (i / rows) * fl.rq + i % rows;
     for (int i = warp; i < terms; i += kWarps) {
       // log2-sum-exp2 of one row of logits by one warp: running (max, sum) per lane, merged in a fixed order
       const float* z = fl.logits + ((long long)(i / rows) * fl.rq + i % rows) * s.total_tokens + tok0;
@@ -139,7 +142,7 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
 #pragma unroll
         for (int u = 0; u < 16; ++u) {
           const int i = i0 + u;
-          v[u] = i < terms ? z[((long long)(i / rows) * fl.rq + i % rows) * s.total_tokens] : -INFINITY;
+          v[u] = i < terms ? z[(long long)term_row[i] * s.total_tokens] : -INFINITY;
         }
 #pragma unroll
         for (int u = 0; u < 16; ++u)
@@ -350,7 +353,7 @@ cudaError_t launch_select(const Shapes& s, const Workspace& w, const float* scor
 // from the logits in the workspace.
 bool narrow_tail_applies(const Shapes& s) {
   const size_t smem = sizeof(SelectShared) + ((size_t)s.max_seqlen + s.max_seqlen / 32 + 1) * sizeof(unsigned) +
-                      (size_t)s.hq * s.max_qlen * sizeof(float);
+                      (size_t)s.hq * s.max_qlen * (sizeof(float) + sizeof(int));
   // one block per sequence does all of it: worth it only while a sequence is short (measured: up to about 1k tokens)
   return s.max_qlen >= 1 && s.max_qlen <= kNarrowMaxRows && s.max_seqlen >= 1 && s.max_seqlen <= 1024 && smem <= 200 * 1024;
 }
@@ -360,7 +363,7 @@ cudaError_t launch_narrow_tail(const Shapes& s, const float* logits, int rq, flo
                                const int32_t* q_idx, const int32_t* cu_qlens, int32_t* keep_idx, int32_t* cu_keep,
                                int32_t* device_status, cudaStream_t stream) {
   const size_t smem = sizeof(SelectShared) + ((size_t)s.max_seqlen + s.max_seqlen / 32 + 1) * sizeof(unsigned) +
-                      (size_t)s.hq * rq * sizeof(float);
+                      (size_t)s.hq * rq * (sizeof(float) + sizeof(int));  // keys, log-sum-exp per term, term offsets
   cudaError_t e = cudaFuncSetAttribute(select_topk_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
   if (e != cudaSuccess) return e;
   e = launch_chained(select_topk_kernel<true, true>, dim3(s.batch), dim3(kThreads), smem, stream, s, (const float*)nullptr,
