@@ -252,7 +252,7 @@ __global__ void __launch_bounds__(kFinalizeThreads) score_narrow_finalize_kernel
                                                                                  const float* __restrict__ logits, int rq,
                                                                                  const float* __restrict__ lse,
                                                                                  float* __restrict__ scores) {
-  extern __shared__ float lse_sh[];  // [Hq][rows]
+  extern __shared__ float lse_sh[];  // [Hq][rows], then the term offsets
   pdl_trigger();
   pdl_wait();
   pdl_acquire(logits);
@@ -262,25 +262,28 @@ __global__ void __launch_bounds__(kFinalizeThreads) score_narrow_finalize_kernel
   if ((int)(blockIdx.x * blockDim.x) >= n) return;
   const int row0 = cu_qlens[b], all_rows = cu_qlens[b + 1] - row0, rows = min(all_rows, rq);
   const int terms = s.hq * rows;
+  // where term i's logits start, in units of N floats: worked out once per block (no integer division per logit below)
+  int* term_row = reinterpret_cast<int*>(lse_sh + s.hq * rq);
   for (int i = threadIdx.x; i < terms; i += blockDim.x) {
     const int head = i / rows, r = i % rows;
     lse_sh[i] = lse[(long long)(row0 + r) * s.hq + head];
+    term_row[i] = head * rq + r;
   }
   __syncthreads();
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   if (j >= n) return;
-  // Term i = (head, row) in head-major order; eight loads in flight, one running sum in that fixed order.
+  // Term i = (head, row) in head-major order; sixteen loads in flight, one running sum in that fixed order.
   const float* z = logits + tok0 + j;
   float total = 0.f;
-  for (int i0 = 0; i0 < terms; i0 += 8) {
-    float v[8];
+  for (int i0 = 0; i0 < terms; i0 += 16) {
+    float v[16];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
+    for (int u = 0; u < 16; ++u) {
       const int i = i0 + u;
-      v[u] = i < terms ? z[((long long)(i / rows) * rq + i % rows) * s.total_tokens] : -INFINITY;
+      v[u] = i < terms ? z[(long long)term_row[i] * s.total_tokens] : -INFINITY;
     }
 #pragma unroll
-    for (int u = 0; u < 8; ++u)
+    for (int u = 0; u < 16; ++u)
       if (i0 + u < terms) total += exp2f(v[u] - lse_sh[i0 + u]);
   }
   scores[tok0 + j] = all_rows > 0 ? total / ((float)s.hq * (float)all_rows) : 0.f;
@@ -354,7 +357,7 @@ cudaError_t launch_score_narrow(const Shapes& s, const Workspace& w, const void*
   if (e != cudaSuccess) return e;
   if ((e = launch_chained(score_narrow_finalize_kernel, dim3((s.max_seqlen + kFinalizeThreads - 1) / kFinalizeThreads, s.batch),
                           dim3(kFinalizeThreads),
-                          s.hq * rq * sizeof(float), stream, s, cu_qlens, cu_seqlens, (const float*)logits, rq, (const float*)lse,
+                          s.hq * rq * (sizeof(float) + sizeof(int)), stream, s, cu_qlens, cu_seqlens, (const float*)logits, rq, (const float*)lse,
                           scores_out)) != cudaSuccess)
     return e;
   count_launches((lse_in ? 0 : 1) + 1);  // the lse import counts itself

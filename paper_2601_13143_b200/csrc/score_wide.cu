@@ -725,12 +725,16 @@ __global__ void __launch_bounds__(kFinalizeThreads) score_wide_finalize_kernel(S
   const int terms = s.hkv * row_chunks;
   const float* col = partial + tok0 + j;
   float total = 0.f;
+  int g = 0, rc = 0;  // (KV head, row chunk) of the next term, stepped along instead of divided out
   for (int i0 = 0; i0 < terms; i0 += 8) {
     float v[8];
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-      const int i = i0 + u;
-      v[u] = i < terms ? col[(long long)((i / row_chunks) * rc_max + i % row_chunks) * s.total_tokens] : 0.f;
+      v[u] = i0 + u < terms ? col[(long long)(g * rc_max + rc) * s.total_tokens] : 0.f;
+      if (++rc == row_chunks) {
+        rc = 0;
+        ++g;
+      }
     }
 #pragma unroll
     for (int u = 0; u < 8; ++u) total += v[u];
