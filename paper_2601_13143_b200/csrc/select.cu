@@ -5,7 +5,9 @@
 // by an MSB-first radix select over the bits in which the keys of the sequence actually differ
 // (the common leading bits come from a min/max reduction; softmax scores share most of their
 // exponent, so without this the first histogram would pile into a handful of bins): at most three
-// passes of 11-bit digits, shared-memory histograms, a block-wide suffix scan to pick the bin.
+// passes of 11-bit digits, shared-memory histograms, a block-wide suffix scan to pick the bin; as soon
+// as the chosen bin holds at most 128 keys (usually after the first pass) they are collected and T is
+// the one whose rank among them is the wanted one, which saves the remaining passes.
 // A single blocked prefix scan in index order then keeps every key above T plus the first
 // (k - #above) keys equal to T: ties go to the lower index and survivors come out ascending, which
 // is exactly the order the gather that follows needs.  Integer work throughout: the result is a
@@ -22,6 +24,7 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kDigitBits = 11;
 constexpr int kBins = 1 << kDigitBits;
 constexpr unsigned kProtectedKey = 0xFFFFFFFFu;
+constexpr int kDirectMax = 128;  // a bucket of at most this many keys is finished by counting ranks, not by more passes
 
 // fp32 -> uint32 with the same ordering as the float comparison (-0 and +0 compare equal).
 __device__ __forceinline__ unsigned order_key(float x) {
@@ -38,6 +41,9 @@ struct SelectShared {
   int remaining;        // how many more keys (from the top of the current bucket) are still to take
   int base;             // output offset of this sequence
   int protected_count;
+  int bucket;           // how many keys the chosen bin of the last pass holds
+  int list_n;           // direct finish: the keys of a small bucket, in no particular order
+  unsigned list[kDirectMax];
 };
 
 // Shared-memory slot of key j: one word of padding per 32 keeps both the strided and the blocked
@@ -275,9 +281,39 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
         const unsigned bin = 2 * tid + (upper ? 1 : 0);
         sh.prefix = prefix | (bin << shift);
         sh.remaining = (int)(rem - above_me - (upper ? 0u : h1));
+        sh.bucket = (int)(upper ? h1 : h0);
+        sh.list_n = 0;
       }
       __syncthreads();
       bits_left = shift;
+      if (bits_left > 0 && sh.bucket <= kDirectMax) {
+        // Few keys left in the bucket (the usual case after the first pass): collect them and let each find its
+        // rank among them; the one whose rank range covers `remaining` is the threshold.
+        const unsigned want = sh.prefix >> bits_left;
+        for (int rd = 0; rd < rounds; ++rd) {
+          const int j = rd * kThreads + tid;
+          const unsigned key = j < n ? keys[slot<kKeysInShared>(j)] : kProtectedKey;
+          if (key != kProtectedKey && (key >> bits_left) == want) sh.list[atomicAdd(&sh.list_n, 1)] = key;
+        }
+        __syncthreads();
+        const int count = sh.list_n, rem_in = sh.remaining;
+        __syncthreads();  // everyone has read `remaining` before an owner rewrites it
+        if (tid < count) {
+          const unsigned mine = sh.list[tid];
+          int above = 0, not_below = 0;
+          for (int i = 0; i < count; ++i) {
+            const unsigned other = sh.list[i];
+            above += other > mine;
+            not_below += other >= mine;
+          }
+          if (above < rem_in && rem_in <= not_below) {  // equal keys all write the same two values
+            sh.prefix = mine;
+            sh.remaining = rem_in - above;
+          }
+        }
+        __syncthreads();
+        bits_left = 0;
+      }
     }
     T = sh.prefix;
     need_eq = sh.remaining;
