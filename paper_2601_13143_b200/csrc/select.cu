@@ -5,8 +5,8 @@
 // by an MSB-first radix select over the bits in which the keys of the sequence actually differ
 // (the common leading bits come from a min/max reduction; softmax scores share most of their
 // exponent, so without this the first histogram would pile into a handful of bins): at most three
-// passes of 11-bit digits, shared-memory histograms, a block-wide suffix scan to pick the bin; as soon
-// as the chosen bin holds at most 128 keys (usually after the first pass) they are collected and T is
+// passes of 13-bit digits (11-bit ones for sequences of at most 2,048 tokens), shared-memory histograms, a block-wide suffix scan to pick the bin; as soon
+// as the chosen bin holds at most 256 keys (usually after the first pass) they are collected and T is
 // the one whose rank among them is the wanted one, which saves the remaining passes.
 // A single blocked prefix scan in index order then keeps every key above T plus the first
 // (k - #above) keys equal to T: ties go to the lower index and survivors come out ascending, which
@@ -21,10 +21,12 @@ namespace {
 
 constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
-constexpr int kDigitBits = 11;
+constexpr int kDigitBits = 13;  // long sequences; short ones (kShortKeys or fewer) take kShortDigitBits, their passes being cheap
+constexpr int kShortDigitBits = 11, kShortKeys = 2048;
 constexpr int kBins = 1 << kDigitBits;
+constexpr int kBinsPerThread = kBins / kThreads;  // bins one thread owns in the suffix scan, at most
 constexpr unsigned kProtectedKey = 0xFFFFFFFFu;
-constexpr int kDirectMax = 128;  // a bucket of at most this many keys is finished by counting ranks, not by more passes
+constexpr int kDirectMax = 256;  // a bucket of at most this many keys is finished by counting ranks, not by more passes
 
 // fp32 -> uint32 with the same ordering as the float comparison (-0 and +0 compare equal).
 __device__ __forceinline__ unsigned order_key(float x) {
@@ -233,8 +235,10 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
       sh.remaining = k - n_protected;
     }
     while (bits_left > 0) {
-      const int width = min(kDigitBits, bits_left), shift = bits_left - width;
-      for (int i = tid; i < kBins; i += kThreads) sh.hist[i] = 0;
+      const int digit_bits = n > kShortKeys ? kDigitBits : kShortDigitBits;
+      const int per_thread = (1 << digit_bits) / kThreads;  // 8 or 2 (uniform)
+      const int width = min(digit_bits, bits_left), shift = bits_left - width;
+      for (int i = tid; i < (1 << digit_bits); i += kThreads) sh.hist[i] = 0;
       __syncthreads();
       const unsigned prefix = sh.prefix;
       const unsigned digit_mask = (1u << width) - 1u;
@@ -254,9 +258,17 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
         }
       }
       __syncthreads();
-      // Suffix sums over the bins, two bins per thread, to find the bin holding the wanted key.
-      const unsigned h0 = sh.hist[2 * tid], h1 = sh.hist[2 * tid + 1];
-      unsigned incl = h0 + h1;  // inclusive suffix sum over threads (higher threads = larger digits)
+      // Suffix sums over the bins, per_thread consecutive bins per thread, to find the bin holding the wanted key.
+      unsigned h[kBinsPerThread];
+      unsigned own = 0;
+#pragma unroll
+      for (int i = 0; i < kBinsPerThread; i += 2) {
+        uint2 q = make_uint2(0u, 0u);
+        if (i < per_thread) q = *reinterpret_cast<const uint2*>(&sh.hist[per_thread * tid + i]);
+        h[i] = q.x; h[i + 1] = q.y;
+        own += q.x + q.y;
+      }
+      unsigned incl = own;  // inclusive suffix sum over threads (higher threads = larger digits)
 #pragma unroll
       for (int d = 1; d < 32; d <<= 1) {
         const unsigned t = __shfl_down_sync(0xFFFFFFFFu, incl, d);
@@ -273,16 +285,21 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
         if (lane + d < 32) suffix += t;
       }
       const unsigned above_warp = __shfl_sync(0xFFFFFFFFu, suffix - own_total, warp);
-      const unsigned above_me = above_warp + incl - (h0 + h1);  // keys in bins above this thread's two
+      const unsigned above_me = above_warp + incl - own;  // keys in bins above this thread's own
       const unsigned rem = (unsigned)sh.remaining;
       __syncthreads();  // everyone has read `remaining` before the one owner rewrites it
-      if (above_me < rem && rem <= above_me + h0 + h1) {
-        const bool upper = rem <= above_me + h1;
-        const unsigned bin = 2 * tid + (upper ? 1 : 0);
-        sh.prefix = prefix | (bin << shift);
-        sh.remaining = (int)(rem - above_me - (upper ? 0u : h1));
-        sh.bucket = (int)(upper ? h1 : h0);
-        sh.list_n = 0;
+      if (above_me < rem && rem <= above_me + own) {
+        unsigned above = above_me;  // walk this thread's bins from the top
+#pragma unroll
+        for (int i = kBinsPerThread - 1; i >= 0; --i) {
+          if (i < per_thread && above < rem && rem <= above + h[i]) {
+            sh.prefix = prefix | ((unsigned)(per_thread * tid + i) << shift);
+            sh.remaining = (int)(rem - above);
+            sh.bucket = (int)h[i];
+            sh.list_n = 0;
+          }
+          above += h[i];
+        }
       }
       __syncthreads();
       bits_left = shift;
