@@ -115,6 +115,12 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 // may otherwise hoist loads through a `const __restrict__` pointer above the wait (it is entitled to
 // assume nobody writes such data while the kernel runs).
 #define pdl_acquire(ptr) asm volatile("" : "+l"(ptr) : : "memory")
+// ... and must never be read through the non-coherent path (ld.global.nc, which __ldg forces): such a load can
+// be served from a line this SM cached during an earlier launch, before the predecessor rewrote it (seen with a
+// kernel that started early under programmatic launch and re-read a buffer of the previous call).  chain_load
+// reads through L2.
+template <typename T>
+__device__ __forceinline__ T chain_load(const T* p) { return __ldcg(p); }
 
 template <typename... KArgs, typename... Args>
 cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {

@@ -529,6 +529,45 @@ def test_prune_random_shapes(seed):
     assert stats["device_status"] & ~fastav.FASTAV_DEV_PROTECT_OVERFLOW == 0
 
 
+@pytest.mark.parametrize("lens,rows,hq,hkv,d", [
+    ([364, 2049, 80, 300], [23, 41, 44, 2], 2, 2, 128),      # tensor-core score, register-resident select
+    ([900, 512, 33], [1, 2, 1], 8, 2, 64),                   # few rows, short: logits + one fused tail kernel
+    ([5000, 3000], [1, 1], 28, 4, 128),                      # few rows, long: logits, statistics, finalize, select
+    ([20000, 100], [40, 3], 4, 2, 64),                       # keys in shared memory (longer than the register kernel takes)
+    ([70000], [8], 4, 1, 64),                                # keys in the workspace
+])
+def test_prune_never_reads_what_an_earlier_call_left_behind(lens, rows, hq, hkv, d):
+    """Kernels of one call start before their predecessors have finished (programmatic launch).  Every buffer a
+    kernel of the chain reads from another is overwritten with poison between calls: a read that comes too
+    early, or from a line cached during the previous call, changes the result."""
+    p = W.random_problem(seed=len(lens) + hq, lens=lens, rows=rows, keeps=[n // 3 + 1 for n in lens], num_q_heads=hq,
+                         num_kv_heads=hkv, head_dim=d, hidden=64)
+    buf = parity.to_device(p)
+    buf.prune()
+    torch.cuda.synchronize()
+    ref = parity.oracle_prune(p)
+    parity.check_fused_against_oracle(p, buf, ref, what=f"lens={lens}")
+    names = ("scores", "keep_idx", "cu_keep", "hidden_out", "k_out", "v_out", "pos_out")
+    first = {k: getattr(buf, k).clone() for k in names}
+    for rep in range(25):
+        buf.scores.fill_(float("nan"))
+        buf.workspace.fill_(0xFF)
+        buf.keep_idx.fill_(-7)
+        buf.cu_keep.fill_(-7)
+        for t in (buf.hidden_out, buf.k_out, buf.v_out):
+            t.view(torch.int16).fill_(0x7FC1)
+        buf.pos_out.fill_(-1)
+        buf.prune()
+        torch.cuda.synchronize()
+        for k in names:
+            a, b = first[k], getattr(buf, k)
+            if a.dtype == torch.float32:
+                a, b = a.view(torch.int32), b.view(torch.int32)
+            elif a.dtype == torch.bfloat16:
+                a, b = a.view(torch.int16), b.view(torch.int16)
+            assert torch.equal(a, b), f"repetition {rep}: {k} differs from the first call"
+
+
 def test_prune_with_protect_mask_keeps_all_text_tokens():
     w = W.WORKLOADS["c1_tiny"]
     p = W.make_stage(w, 0)
