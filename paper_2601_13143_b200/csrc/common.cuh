@@ -121,6 +121,10 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 // reads through L2.
 template <typename T>
 __device__ __forceinline__ T chain_load(const T* p) { return __ldcg(p); }
+// The same for values read many times (a table that is searched): an ordinary coherent load that may stay in L1,
+// spelled out so that it can never turn into the non-coherent form.
+template <typename T>
+__device__ __forceinline__ T chain_load_cached(const T* p) { return __ldca(p); }
 
 template <typename... KArgs, typename... Args>
 cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {

@@ -59,16 +59,16 @@ __global__ void __launch_bounds__(kThreads) compact_rows_kernel(Shapes s, RowStr
   const int n_chunks = n_hidden + n_k + n_v;
   const int head_shift = (s.dim == 128) ? 4 : 3;
   const bool global_idx = (s.flags & FASTAV_KEEP_IDX_GLOBAL) != 0;
-  int rows = cu_keep[s.batch];
+  int rows = chain_load_cached(cu_keep + s.batch);
   if (rows > s.total_keep) rows = s.total_keep;  // never write past the caller's buffers
 
   for (int row = blockIdx.x; row < rows; row += gridDim.x) {
     int lo = 0, hi = s.batch;  // largest b with cu_keep[b] <= row
     while (hi - lo > 1) {
       const int mid = (lo + hi) >> 1;
-      if (cu_keep[mid] <= row) lo = mid; else hi = mid;
+      if (chain_load_cached(cu_keep + mid) <= row) lo = mid; else hi = mid;
     }
-    const long long src = global_idx ? (long long)keep_idx[row] : (long long)cu_seqlens[lo] + keep_idx[row];
+    const long long src = (global_idx ? 0ll : (long long)cu_seqlens[lo]) + chain_load(keep_idx + row);
     const long long dst = row;
     if (src < cu_seqlens[lo] || src >= cu_seqlens[lo + 1]) {  // an index outside its sequence: skip the row, report
       if (threadIdx.x == 0 && device_status) atomicOr(device_status, FASTAV_DEV_BAD_INDEX);
@@ -192,7 +192,7 @@ compact_rows_bulk_kernel(Shapes s, RowStreams t, const int32_t* __restrict__ kee
   pdl_wait();  // keep_idx and cu_keep are the previous kernel's output
   pdl_acquire(keep_idx);
   pdl_acquire(cu_keep);
-  int rows = cu_keep[s.batch];
+  int rows = chain_load_cached(cu_keep + s.batch);
   if (rows > s.total_keep) rows = s.total_keep;  // never write past the caller's buffers
   const int first = blockIdx.x * warps + warp, step = gridDim.x * warps;
   const int my_rows = first < rows ? (rows - first + step - 1) / step : 0;
@@ -203,9 +203,9 @@ compact_rows_bulk_kernel(Shapes s, RowStreams t, const int32_t* __restrict__ kee
     int lo = 0, hi = s.batch;  // largest b with cu_keep[b] <= row
     while (hi - lo > 1) {
       const int mid = (lo + hi) >> 1;
-      if (cu_keep[mid] <= row) lo = mid; else hi = mid;
+      if (chain_load_cached(cu_keep + mid) <= row) lo = mid; else hi = mid;
     }
-    const long long src = global_idx ? (long long)keep_idx[row] : (long long)cu_seqlens[lo] + keep_idx[row];
+    const long long src = (global_idx ? 0ll : (long long)cu_seqlens[lo]) + chain_load(keep_idx + row);
     if (src < cu_seqlens[lo] || src >= cu_seqlens[lo + 1]) {
       if (lane == 0 && device_status) atomicOr(device_status, FASTAV_DEV_BAD_INDEX);
       return -1;

@@ -130,7 +130,7 @@ score_narrow_logits_kernel(Shapes s, const uint16_t* __restrict__ q, const int32
       const int f = pass0 + i;
       uint4 raw = make_uint4(0, 0, 0, 0);
       if (f < flat_rows)
-        raw = __ldg(reinterpret_cast<const uint4*>(q + (long long)(row0 + f / s.group) * s.q_st +
+        raw = chain_load(reinterpret_cast<const uint4*>(q + (long long)(row0 + f / s.group) * s.q_st +
                                                    (long long)(head * s.group + f % s.group) * s.q_sh + lane * 8));
       unpack8(raw, qv[i]);
     }
@@ -213,7 +213,7 @@ __global__ void __launch_bounds__(256) score_narrow_stats_kernel(Shapes s, const
   for (int j0 = threadIdx.x; j0 < n; j0 += 256 * 4) {
     float v[4];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) v[u] = j0 + u * 256 < n ? z[j0 + u * 256] : -INFINITY;
+    for (int u = 0; u < 4; ++u) v[u] = j0 + u * 256 < n ? chain_load(z + j0 + u * 256) : -INFINITY;
     const float m_new = fmaxf(fmaxf(m, fmaxf(v[0], v[1])), fmaxf(v[2], v[3]));
     if (m_new > -INFINITY) {
       l = l * exp2f(m - m_new);
@@ -266,7 +266,7 @@ __global__ void __launch_bounds__(kFinalizeThreads) score_narrow_finalize_kernel
   int* term_row = reinterpret_cast<int*>(lse_sh + s.hq * rq);
   for (int i = threadIdx.x; i < terms; i += blockDim.x) {
     const int head = i / rows, r = i % rows;
-    lse_sh[i] = lse[(long long)(row0 + r) * s.hq + head];
+    lse_sh[i] = chain_load(lse + (long long)(row0 + r) * s.hq + head);
     term_row[i] = head * rq + r;
   }
   __syncthreads();
@@ -280,7 +280,7 @@ __global__ void __launch_bounds__(kFinalizeThreads) score_narrow_finalize_kernel
 #pragma unroll
     for (int u = 0; u < 16; ++u) {
       const int i = i0 + u;
-      v[u] = i < terms ? z[(long long)term_row[i] * s.total_tokens] : -INFINITY;
+      v[u] = i < terms ? chain_load(z + (long long)term_row[i] * s.total_tokens) : -INFINITY;
     }
 #pragma unroll
     for (int u = 0; u < 16; ++u)

@@ -619,7 +619,7 @@ score_wide_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
             int lim = -1;
             if (c < my_cols) {
               const int r = f / s.group;
-              nl = -lse[(long long)(un.row0 + r) * s.hq + un.g * s.group + f % s.group];
+              nl = -chain_load(lse + (long long)(un.row0 + r) * s.hq + un.g * s.group + f % s.group);
               lim = causal ? q_idx[un.row0 + r] : INT_MAX;
               min_limit = min(min_limit, lim);
             }
@@ -691,13 +691,13 @@ __global__ void __launch_bounds__(256) score_wide_merge_kernel(Shapes s, const i
   const int chunks = 2 * ((n + chunk_keys - 1) / chunk_keys);  // one entry per 64-key half of every tile run
   const float2* mine = stats + (long long)w * stat_chunks;
   float m = -INFINITY;
-  for (int t = lane; t < chunks; t += 32) m = fmaxf(m, mine[t].x);
+  for (int t = lane; t < chunks; t += 32) m = fmaxf(m, chain_load(mine + t).x);
 #pragma unroll
   for (int d = 16; d; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, d));
   float l = 0.f;
   if (m > -INFINITY)
     for (int t = lane; t < chunks; t += 32) {
-      const float2 v = mine[t];
+      const float2 v = chain_load(mine + t);
       if (v.x > -INFINITY) l += v.y * exp2f(v.x - m);
     }
 #pragma unroll
@@ -730,7 +730,7 @@ __global__ void __launch_bounds__(kFinalizeThreads) score_wide_finalize_kernel(S
     float v[8];
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-      v[u] = i0 + u < terms ? col[(long long)(g * rc_max + rc) * s.total_tokens] : 0.f;
+      v[u] = i0 + u < terms ? chain_load(col + (long long)(g * rc_max + rc) * s.total_tokens) : 0.f;
       if (++rc == row_chunks) {
         rc = 0;
         ++g;

@@ -122,7 +122,7 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
       for (int j0 = lane; j0 < n; j0 += 512) {  // sixteen loads in flight per lane: at most two trips for 1,024 tokens
         float v[16];
 #pragma unroll
-        for (int u = 0; u < 16; ++u) v[u] = j0 + 32 * u < n ? z[j0 + 32 * u] : -INFINITY;
+        for (int u = 0; u < 16; ++u) v[u] = j0 + 32 * u < n ? chain_load(z + j0 + 32 * u) : -INFINITY;
         float m_new = m;
 #pragma unroll
         for (int u = 0; u < 16; ++u) m_new = fmaxf(m_new, v[u]);
@@ -150,7 +150,7 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
 #pragma unroll
         for (int u = 0; u < 16; ++u) {
           const int i = i0 + u;
-          v[u] = i < terms ? z[(long long)term_row[i] * s.total_tokens] : -INFINITY;
+          v[u] = i < terms ? chain_load(z + (long long)term_row[i] * s.total_tokens) : -INFINITY;
         }
 #pragma unroll
         for (int u = 0; u < 16; ++u)
@@ -764,14 +764,15 @@ __global__ void __launch_bounds__(kThreads) mask_emit_kernel(Shapes s, const uin
   if (tid == 0) base_sh = 0;
   __syncthreads();
   int part = 0;
-  for (int i = tid; i < b; i += kThreads) part += counts[i];
+  for (int i = tid; i < b; i += kThreads) part += chain_load(counts + i);
   if (part) atomicAdd(&base_sh, part);
   __syncthreads();
   const int base = base_sh;
   if (tid == 0) {
-    cu_keep[b + 1] = min(base + counts[b], s.total_keep);
+    const int mine = chain_load(counts + b);
+    cu_keep[b + 1] = min(base + mine, s.total_keep);
     if (b == 0) cu_keep[0] = 0;
-    if (base + counts[b] > s.total_keep && device_status) atomicOr(device_status, FASTAV_DEV_K_CLAMPED);
+    if (base + mine > s.total_keep && device_status) atomicOr(device_status, FASTAV_DEV_K_CLAMPED);
   }
   const bool global_idx = (s.flags & FASTAV_KEEP_IDX_GLOBAL) != 0;
   const int per = (n + kThreads - 1) / kThreads;
