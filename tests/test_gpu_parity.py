@@ -256,7 +256,7 @@ def test_select_sequence_longer_than_shared_memory():
 
 @pytest.mark.parametrize("longest", [2048, 2049, 4097, 8200, 16384, 40_000, 131_072, 131_073])
 def test_select_long_sequences_in_ragged_batches(longest):
-    """Keep lists of long sequences (keys in shared memory up to about 57k tokens, in the workspace above)
+    """Keep lists of long sequences (keys in shared memory up to about 50k tokens, in the workspace above)
     with short and empty sequences in the same batch: heavy ties, protected tokens and scored rows anywhere,
     a long run of equal scores, nearly everything or nearly nothing kept."""
     rng = np.random.default_rng(longest)
