@@ -548,8 +548,24 @@ def test_prune_never_reads_what_an_earlier_call_left_behind(lens, rows, hq, hkv,
     ref = parity.oracle_prune(p)
     parity.check_fused_against_oracle(p, buf, ref, what=f"lens={lens}")
     names = ("scores", "keep_idx", "cu_keep", "hidden_out", "k_out", "v_out", "pos_out")
-    first = {k: getattr(buf, k).clone() for k in names}
-    for rep in range(25):
+
+    def run(fused):
+        if fused:
+            buf.prune()
+        else:                      # the same three steps as separate calls: they chain on the stream in the same way
+            buf.score()
+            buf.select()
+            buf.compact()
+        torch.cuda.synchronize()
+
+    def bits(t):
+        return t.view(torch.int32) if t.dtype == torch.float32 else t.view(torch.int16) if t.dtype == torch.bfloat16 else t
+
+    first = {}
+    for fused in (True, False):    # the two routes may round the scores differently; each is compared with itself
+        run(fused)
+        first[fused] = {k: getattr(buf, k).clone() for k in names}
+    for rep in range(30):
         buf.scores.fill_(float("nan"))
         buf.workspace.fill_(0xFF)
         buf.keep_idx.fill_(-7)
@@ -557,15 +573,10 @@ def test_prune_never_reads_what_an_earlier_call_left_behind(lens, rows, hq, hkv,
         for t in (buf.hidden_out, buf.k_out, buf.v_out):
             t.view(torch.int16).fill_(0x7FC1)
         buf.pos_out.fill_(-1)
-        buf.prune()
-        torch.cuda.synchronize()
+        fused = rep % 2 == 0
+        run(fused)
         for k in names:
-            a, b = first[k], getattr(buf, k)
-            if a.dtype == torch.float32:
-                a, b = a.view(torch.int32), b.view(torch.int32)
-            elif a.dtype == torch.bfloat16:
-                a, b = a.view(torch.int16), b.view(torch.int16)
-            assert torch.equal(a, b), f"repetition {rep}: {k} differs from the first call"
+            assert torch.equal(bits(first[fused][k]), bits(getattr(buf, k))), f"repetition {rep}: {k} differs from the first call"
 
 
 def test_prune_with_protect_mask_keeps_all_text_tokens():
