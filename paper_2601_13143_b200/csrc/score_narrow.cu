@@ -200,12 +200,13 @@ __global__ void __launch_bounds__(256) score_narrow_stats_kernel(Shapes s, const
                                                                  float* __restrict__ lse) {
   __shared__ float red[8];
   pdl_trigger();
-  pdl_wait();
-  pdl_acquire(logits);
+  // the caller's arrays first: these loads overlap the predecessor's tail
   const int b = blockIdx.y, head = blockIdx.x / rq, r = blockIdx.x % rq;
   const int row0 = cu_qlens[b], rows = min(cu_qlens[b + 1] - row0, rq);
-  if (r >= rows) return;
   const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
+  pdl_wait();
+  pdl_acquire(logits);
+  if (r >= rows) return;
   const float* z = logits + ((long long)head * rq + r) * s.total_tokens + tok0;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   // One pass: every thread keeps a running (max, sum 2^(z - max)) over its strided share, four loads at a time.
@@ -254,14 +255,15 @@ __global__ void __launch_bounds__(kFinalizeThreads) score_narrow_finalize_kernel
                                                                                  float* __restrict__ scores) {
   extern __shared__ float lse_sh[];  // [Hq][rows], then the term offsets
   pdl_trigger();
+  // the caller's arrays first: these loads overlap the predecessor's tail
+  const int b = blockIdx.y;
+  const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
+  const int row0 = cu_qlens[b], all_rows = cu_qlens[b + 1] - row0, rows = min(all_rows, rq);
+  const int terms = s.hq * rows;
   pdl_wait();
   pdl_acquire(logits);
   pdl_acquire(lse);
-  const int b = blockIdx.y;
-  const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
   if ((int)(blockIdx.x * blockDim.x) >= n) return;
-  const int row0 = cu_qlens[b], all_rows = cu_qlens[b + 1] - row0, rows = min(all_rows, rq);
-  const int terms = s.hq * rows;
   // where term i's logits start, in units of N floats: worked out once per block (no integer division per logit below)
   int* term_row = reinterpret_cast<int*>(lse_sh + s.hq * rq);
   for (int i = threadIdx.x; i < terms; i += blockDim.x) {

@@ -677,29 +677,38 @@ __global__ void __launch_bounds__(256) score_wide_merge_kernel(Shapes s, const i
                                                                const float2* __restrict__ stats, int stat_chunks,
                                                                int chunk_keys, float* __restrict__ lse) {
   pdl_trigger();
+  // which sequence this warp's row belongs to: from the caller's arrays, so before the wait
+  const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  const bool active = w < s.total_q * s.hq;
+  int chunks = 0;
+  if (active) {
+    const int row = w / s.hq;
+    int lo = 0, hi = s.batch;
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (cu_qlens[mid] <= row) lo = mid; else hi = mid;
+    }
+    const int n = cu_seqlens[lo + 1] - cu_seqlens[lo];
+    chunks = 2 * ((n + chunk_keys - 1) / chunk_keys);  // one entry per 64-key half of every tile run
+  }
   pdl_wait();
   pdl_acquire(stats);
-  const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (w >= s.total_q * s.hq) return;
-  const int row = w / s.hq;
-  int lo = 0, hi = s.batch;
-  while (hi - lo > 1) {
-    const int mid = (lo + hi) >> 1;
-    if (cu_qlens[mid] <= row) lo = mid; else hi = mid;
-  }
-  const int n = cu_seqlens[lo + 1] - cu_seqlens[lo];
-  const int chunks = 2 * ((n + chunk_keys - 1) / chunk_keys);  // one entry per 64-key half of every tile run
+  if (!active) return;
   const float2* mine = stats + (long long)w * stat_chunks;
-  float m = -INFINITY;
-  for (int t = lane; t < chunks; t += 32) m = fmaxf(m, chain_load(mine + t).x);
+  // the first 32 entries stay in a register (usually all of them); the rest, if any, is read twice
+  const float2 first = lane < chunks ? chain_load(mine + lane) : make_float2(-INFINITY, 0.f);
+  float m = first.x;
+  for (int t = lane + 32; t < chunks; t += 32) m = fmaxf(m, chain_load(mine + t).x);
 #pragma unroll
   for (int d = 16; d; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, d));
   float l = 0.f;
-  if (m > -INFINITY)
-    for (int t = lane; t < chunks; t += 32) {
+  if (m > -INFINITY) {
+    if (first.x > -INFINITY) l = first.y * exp2f(first.x - m);
+    for (int t = lane + 32; t < chunks; t += 32) {
       const float2 v = chain_load(mine + t);
       if (v.x > -INFINITY) l += v.y * exp2f(v.x - m);
     }
+  }
 #pragma unroll
   for (int d = 16; d; d >>= 1) l += __shfl_xor_sync(0xFFFFFFFFu, l, d);
   if (lane == 0) lse[w] = (l > 0.f) ? m + log2f(l) : INFINITY;  // a row that sees no key contributes 0
