@@ -52,6 +52,14 @@ extern "C" {
 #define FASTAV_CAUSAL 1u              /* scored row r sees keys j <= q_idx[r] only (the model's own mask) */
 #define FASTAV_PROTECT_QUERY_ROWS 2u  /* the scored rows' tokens always survive (and count toward k_b) */
 #define FASTAV_KEEP_IDX_GLOBAL 4u     /* keep_idx holds indices into the packed batch, not sequence-local ones */
+#define FASTAV_CHAIN_CALLS 0x1000u    /* The index arrays of this call (cu_seqlens, cu_qlens, q_idx, keep_counts, protect) were
+                                         complete before the work that precedes the call on the stream was enqueued (e.g.
+                                         uploaded once for all pruning layers: the survivor counts are known on the host).
+                                         The call's first kernel may then start, and read them, while that earlier work is
+                                         still running, which hides its set-up behind the previous call's last kernel.
+                                         Without the flag the first kernel starts when all earlier work has completed, so
+                                         the arrays may be what the previous kernel wrote (a cu_keep_out used as the next
+                                         cu_seqlens).  q, k, v, hidden, pos, scores and keep lists are never read early. */
 #define FASTAV_SELECT_LOWEST 0x800u   /* fastav_select keeps the k_b LOWEST-scoring tokens instead: the "prune the most attended
                                          tokens" control of the paper's ablations (Tables 2 and 3, "Top attentive") */
 

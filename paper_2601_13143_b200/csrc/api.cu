@@ -213,6 +213,7 @@ int32_t fastav_score(const fastav_params* params, const void* q, const int32_t* 
                      void* workspace, size_t workspace_bytes, int32_t* device_status, void* stream) {
   int32_t rc = check_params(params);
   if (rc != FASTAV_OK) return rc;
+  chain_begin(params->flags);
   if ((rc = check_score_args(params, q, q_idx, cu_qlens, k, cu_seqlens, scores_out)) != FASTAV_OK) return rc;
   const Workspace w = plan_workspace(*params);
   if ((rc = check_workspace(w, workspace, workspace_bytes)) != FASTAV_OK) return rc;
@@ -229,6 +230,7 @@ int32_t fastav_select(const fastav_params* params, const float* scores, const in
                       size_t workspace_bytes, int32_t* device_status, void* stream) {
   int32_t rc = check_params(params);
   if (rc != FASTAV_OK) return rc;
+  chain_begin(params->flags);
   if ((rc = check_select_args(params, scores, cu_seqlens, keep_counts, q_idx, cu_qlens, keep_idx_out, cu_keep_out)) != FASTAV_OK) return rc;
   const Workspace w = plan_workspace(*params);
   if ((rc = check_workspace(w, workspace, workspace_bytes)) != FASTAV_OK) return rc;
@@ -244,6 +246,7 @@ int32_t fastav_compact(const fastav_params* params, const int32_t* keep_idx, con
                        int32_t* device_status, void* stream) {
   int32_t rc = check_params(params);
   if (rc != FASTAV_OK) return rc;
+  chain_begin(params->flags);
   if ((rc = check_compact_args(params, keep_idx, cu_keep, cu_seqlens, hidden_in, hidden_out, pos_in, pos_out, k_in, k_out,
                                v_in, v_out)) != FASTAV_OK)
     return rc;
@@ -260,6 +263,7 @@ int32_t fastav_prune(const fastav_params* params, const void* q, const int32_t* 
   // Validate everything first so that an error leaves nothing enqueued.
   int32_t rc = check_params(params);
   if (rc != FASTAV_OK) return rc;
+  chain_begin(params->flags);
   if ((rc = check_score_args(params, q, q_idx, cu_qlens, k, cu_seqlens, scores_out)) != FASTAV_OK) return rc;
   if ((rc = check_select_args(params, scores_out, cu_seqlens, keep_counts, q_idx, cu_qlens, keep_idx_out, cu_keep_out)) != FASTAV_OK) return rc;
   if ((rc = check_compact_args(params, keep_idx_out, cu_keep_out, cu_seqlens, hidden_in, hidden_out, pos_in, pos_out, k, k_out,

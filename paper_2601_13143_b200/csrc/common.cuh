@@ -126,6 +126,15 @@ __device__ __forceinline__ T chain_load(const T* p) { return __ldcg(p); }
 template <typename T>
 __device__ __forceinline__ T chain_load_cached(const T* p) { return __ldca(p); }
 
+// The FIRST kernel an entry point launches takes an ordinary stream dependency: it starts only when all earlier
+// work on the stream has completed, so that the arrays the kernels read before their wait (cu_seqlens, cu_qlens,
+// q_idx, keep_counts, protect: possibly the output of the call before, e.g. its cu_keep) are final.  Every later
+// kernel of the call is launched programmatically.  Under FASTAV_CHAIN_CALLS the caller vouches for those arrays
+// and the first kernel is launched programmatically as well.  chain_begin() marks the start of a call (per host
+// thread).
+inline thread_local bool g_chain_head = true;
+inline void chain_begin(uint32_t flags) { g_chain_head = (flags & FASTAV_CHAIN_CALLS) == 0; }
+
 template <typename... KArgs, typename... Args>
 cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {
   cudaLaunchConfig_t cfg = {};
@@ -137,7 +146,8 @@ cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = g_chain_head ? 0 : 1;
+  g_chain_head = false;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 #endif

@@ -802,6 +802,7 @@ __global__ void __launch_bounds__(kThreads) mask_emit_kernel(Shapes s, const uin
 extern "C" int32_t fastav_select_mask(const fastav_params* p, const uint8_t* keep_mask, const int32_t* cu_seqlens,
                                       int32_t* keep_idx_out, int32_t* cu_keep_out, void* workspace, size_t workspace_bytes,
                                       int32_t* device_status, void* stream) {
+  fastav::chain_begin(p ? p->flags : 0u);
   using namespace fastav;
   if (!p || p->batch < 1 || p->total_tokens < 0 || p->total_keep < 0 || p->total_keep > p->total_tokens) return FASTAV_ERR_INVALID_ARG;
   if (!cu_seqlens || !cu_keep_out || (p->total_tokens > 0 && !keep_mask) || (p->total_keep > 0 && !keep_idx_out))
@@ -863,6 +864,7 @@ extern "C" int32_t fastav_select_noalloc(const fastav_params* p, const float* sc
                                          const int32_t* keep_counts, const uint8_t* protect_opt, const int32_t* q_idx,
                                          const int32_t* cu_qlens, int32_t* keep_idx_out, int32_t* cu_keep_out,
                                          int32_t* device_status, void* stream) {
+  fastav::chain_begin(p ? p->flags : 0u);
   using namespace fastav;
   if (!p || p->batch < 1 || p->total_tokens < 0 || p->max_seqlen < 0 || p->max_seqlen > p->total_tokens ||
       p->total_keep < 0 || p->total_keep > p->total_tokens || p->total_q < 0)

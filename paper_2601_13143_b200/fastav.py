@@ -17,6 +17,7 @@ FASTAV_CAUSAL = 1
 FASTAV_PROTECT_QUERY_ROWS = 2
 FASTAV_KEEP_IDX_GLOBAL = 4
 FASTAV_SELECT_LOWEST = 0x800
+FASTAV_CHAIN_CALLS = 0x1000
 
 FASTAV_SCORE_PATH_GENERIC = 0x100
 FASTAV_SCORE_PATH_NARROW = 0x200

@@ -521,7 +521,8 @@ def test_prune_random_shapes(seed):
     path = str(rng.choice(["auto", "auto", "generic", "narrow", "wide"]))
     if not _path_applies(path, [min(r, n) for r, n in zip(rows, lens)], hq, hkv, d):
         path = "auto"
-    buf = parity.to_device(p, protect=protect, extra_flags=SCORE_PATHS[path])
+    chain = fastav.FASTAV_CHAIN_CALLS if rng.random() < 0.5 else 0      # inputs are complete either way
+    buf = parity.to_device(p, protect=protect, extra_flags=SCORE_PATHS[path] | chain)
     buf.prune()
     torch.cuda.synchronize()
     ref = parity.oracle_prune(p, protect=protect)
@@ -536,13 +537,14 @@ def test_prune_random_shapes(seed):
     ([20000, 100], [40, 3], 4, 2, 64),                       # keys in shared memory (longer than the register kernel takes)
     ([70000], [8], 4, 1, 64),                                # keys in the workspace
 ])
-def test_prune_never_reads_what_an_earlier_call_left_behind(lens, rows, hq, hkv, d):
+@pytest.mark.parametrize("chain", [0, fastav.FASTAV_CHAIN_CALLS])
+def test_prune_never_reads_what_an_earlier_call_left_behind(lens, rows, hq, hkv, d, chain):
     """Kernels of one call start before their predecessors have finished (programmatic launch).  Every buffer a
     kernel of the chain reads from another is overwritten with poison between calls: a read that comes too
     early, or from a line cached during the previous call, changes the result."""
     p = W.random_problem(seed=len(lens) + hq, lens=lens, rows=rows, keeps=[n // 3 + 1 for n in lens], num_q_heads=hq,
                          num_kv_heads=hkv, head_dim=d, hidden=64)
-    buf = parity.to_device(p)
+    buf = parity.to_device(p, extra_flags=chain)
     buf.prune()
     torch.cuda.synchronize()
     ref = parity.oracle_prune(p)
@@ -577,6 +579,43 @@ def test_prune_never_reads_what_an_earlier_call_left_behind(lens, rows, hq, hkv,
         run(fused)
         for k in names:
             assert torch.equal(bits(first[fused][k]), bits(getattr(buf, k))), f"repetition {rep}: {k} differs from the first call"
+
+
+@pytest.mark.parametrize("lens,rows1,rows2,hq,hkv,d", [([700, 300, 2049], [40, 8, 16], [1, 1, 1], 8, 2, 64),
+                                                        ([900, 512], [1, 1], [1, 1], 28, 4, 128)])
+def test_second_call_may_take_its_cu_seqlens_from_the_first(lens, rows1, rows2, hq, hkv, d):
+    """Two pruning layers back to back on one stream, the second reading the FIRST call's cu_keep_out as its
+    cu_seqlens and its hidden/pos outputs as inputs (no FASTAV_CHAIN_CALLS: those arrays are written by the call
+    before).  Outputs of the first call are poisoned before every repetition, so a second call that read them too
+    early would see poison."""
+    keeps1 = [n // 2 for n in lens]
+    keeps2 = [k * 3 // 4 for k in keeps1]
+    p1 = W.random_problem(seed=21, lens=lens, rows=rows1, keeps=keeps1, num_q_heads=hq, num_kv_heads=hkv, head_dim=d, hidden=128)
+    p1.protect_rows = True
+    p2 = W.random_problem(seed=22, lens=keeps1, rows=rows2, keeps=keeps2, num_q_heads=hq, num_kv_heads=hkv, head_dim=d, hidden=128)
+    p2.protect_rows = True
+    b1 = parity.to_device(p1)
+    dev = lambda t: t.cuda()
+    b2 = fastav.make_buffers(q=dev(p2.q), q_idx=dev(p2.q_idx), cu_qlens=dev(p2.cu_qlens), k=dev(p2.k), v=dev(p2.v),
+                             cu_seqlens=b1.cu_keep, keep_counts=dev(p2.keep_counts), hidden=b1.hidden_out, pos=b1.pos_out,
+                             softmax_scale=p2.softmax_scale, flags=parity.flags_of(p2), lens=keeps1,
+                             rows=[min(r, n) for r, n in zip(rows2, keeps1)], keeps=keeps2)
+    ref1 = parity.oracle_prune(p1)
+    ref2 = parity.oracle_prune(p2, hidden=torch.from_numpy(ref1["hidden"].view(np.int16)).view(torch.bfloat16),
+                               pos=torch.from_numpy(ref1["pos"]))
+    for rep in range(10):
+        b1.cu_keep.fill_(-7)
+        b1.hidden_out.view(torch.int16).fill_(0x7FC1)
+        b1.pos_out.fill_(-1)
+        b2.scores.fill_(float("nan"))
+        b1.prune()
+        b2.prune()
+        torch.cuda.synchronize()
+        s1 = parity.check_fused_against_oracle(p1, b1, ref1, what=f"first call, repetition {rep}")
+        if s1["ambiguous_differing"] == 0:
+            s2 = parity.check_fused_against_oracle(p2, b2, ref2, hidden=b1.hidden_out.cpu(), pos=b1.pos_out.cpu(),
+                                                   what=f"second call, repetition {rep}")
+            assert s2["device_status"] == 0
 
 
 def test_prune_with_protect_mask_keeps_all_text_tokens():
