@@ -145,6 +145,21 @@ int32_t fastav_score(const fastav_params* params, const void* q, const int32_t* 
                      void* workspace, size_t workspace_bytes, int32_t* device_status, void* stream);
 
 /*
+ * The first sweep alone: log sum exp of every scored row's logits, per head -- what an attention kernel
+ * reports for these rows, in its convention (Section 1: the method needs no attention map, only what a
+ * FlashAttention-style kernel already has):
+ *
+ *   lse_out [total_q, Hq] fp32   natural logarithm of sum_j exp(scale * <q[r,h,:], k[j,h/G,:]>) over the keys
+ *                                row r may see; -inf for a row that sees none
+ *
+ * Handing it back to fastav_score as lse_opt gives the same scores as the self-contained call (to rounding).
+ * Arguments, workspace and errors as for fastav_score.
+ */
+int32_t fastav_lse(const fastav_params* params, const void* q, const int32_t* q_idx, const int32_t* cu_qlens, const void* k,
+                   const int32_t* cu_seqlens, float* lse_out, void* workspace, size_t workspace_bytes, int32_t* device_status,
+                   void* stream);
+
+/*
  * "Tokens with the lowest P% scores are removed" (Section 2.2): per sequence keep the
  * keep_counts[b] highest-scoring tokens; equal scores go to the lower index; protected tokens
  * (protect_opt[j] != 0, and the scored rows' tokens under FASTAV_PROTECT_QUERY_ROWS) rank above

@@ -224,6 +224,27 @@ int32_t fastav_score(const fastav_params* params, const void* q, const int32_t* 
   return e == cudaSuccess ? FASTAV_OK : cuda_failed(e);
 }
 
+int32_t fastav_lse(const fastav_params* params, const void* q, const int32_t* q_idx, const int32_t* cu_qlens, const void* k,
+                   const int32_t* cu_seqlens, float* lse_out, void* workspace, size_t workspace_bytes, int32_t* device_status,
+                   void* stream) {
+  int32_t rc = check_params(params);
+  if (rc != FASTAV_OK) return rc;
+  chain_begin(params->flags);
+  if (!lse_out && params->total_q > 0) return FASTAV_ERR_INVALID_ARG;
+  // the scores pointer only has to be non-null for the shared argument check; nothing is written through it
+  if ((rc = check_score_args(params, q, q_idx, cu_qlens, k, cu_seqlens, lse_out)) != FASTAV_OK) return rc;
+  const Workspace w = plan_workspace(*params);
+  if ((rc = check_workspace(w, workspace, workspace_bytes)) != FASTAV_OK) return rc;
+  const Shapes s = make_shapes(*params);
+  if (!score_path_ok(s)) return FASTAV_ERR_UNSUPPORTED;
+  if (params->total_tokens == 0 || params->total_q == 0) return FASTAV_OK;
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e = launch_score(s, w, q, q_idx, cu_qlens, k, cu_seqlens, nullptr, nullptr, ws, device_status, st);
+  if (e == cudaSuccess) e = launch_lse_export(s, reinterpret_cast<const float*>(ws + w.lse_off), lse_out, st);
+  return e == cudaSuccess ? FASTAV_OK : cuda_failed(e);
+}
+
 int32_t fastav_select(const fastav_params* params, const float* scores, const int32_t* cu_seqlens,
                       const int32_t* keep_counts, const uint8_t* protect_opt, const int32_t* q_idx,
                       const int32_t* cu_qlens, int32_t* keep_idx_out, int32_t* cu_keep_out, void* workspace,

@@ -11,6 +11,7 @@ namespace fastav {
 
 constexpr int kNumSMs = 148;          // B200: 2 dies x 74 SMs; grids are sized in multiples of this
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
 
 // Device-side view of one call's shapes (a trimmed fastav_params, passed by value).
 struct Shapes {
@@ -50,6 +51,8 @@ cudaError_t launch_score_generic(const Shapes& s, const Workspace& w, const void
 // lse_ws[i] = log2(e) * lse_in[i] (the kernels work in base-2 units); a non-finite entry (a row that saw no
 // key) becomes +inf, i.e. the row contributes nothing.
 cudaError_t launch_lse_import(const Shapes& s, const float* lse_in, float* lse_ws, cudaStream_t stream);
+// ... and back: the workspace's statistics as natural-log log-sum-exp [total_q, Hq] (-inf where a row sees no key).
+cudaError_t launch_lse_export(const Shapes& s, const float* lse_ws, float* lse_out, cudaStream_t stream);
 
 // Few scored rows per sequence (the paper's fine stage scores the last token only): matrix-vector path.
 constexpr int kNarrowMaxRows = 4;

@@ -246,6 +246,18 @@ __global__ void __launch_bounds__(256) lse_import_kernel(int count, const float*
   lse_ws[i] = (v == v && fabsf(v) != INFINITY) ? v * kLog2e : INFINITY;
 }
 
+// The way back: log2-sum-exp2 of the workspace -> natural-log log-sum-exp as attention kernels report it
+// (-inf for a row that sees no key).
+__global__ void __launch_bounds__(256) lse_export_kernel(int count, const float* __restrict__ lse_ws, float* __restrict__ lse_out) {
+  pdl_trigger();
+  pdl_wait();
+  pdl_acquire(lse_ws);
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  const float v = chain_load(lse_ws + i);
+  lse_out[i] = v == INFINITY ? -INFINITY : v * kLn2;
+}
+
 template <int DIM>
 cudaError_t run(const Shapes& s, const Workspace& w, const uint16_t* q, const int32_t* q_idx, const int32_t* cu_qlens,
                 const uint16_t* k, const int32_t* cu_seqlens, const float* lse_in, float* scores_out, unsigned char* ws,
@@ -267,10 +279,11 @@ cudaError_t run(const Shapes& s, const Workspace& w, const uint16_t* q, const in
       score_merge_stats_kernel<<<(warps + 7) / 8, 256, 0, stream>>>(s, cu_qlens, cu_seqlens, stats, w.stat_tiles, lse);
       count_launches(2);
     }
+    if (!scores_out) return cudaGetLastError();  // only the statistics were asked for (fastav_lse)
     score_tile_accumulate_kernel<DIM><<<grid, kThreads, smem, stream>>>(s, q, q_idx, cu_qlens, k, cu_seqlens, lse, partial);
     count_launches(1);
   }
-  if (s.max_seqlen > 0) {
+  if (s.max_seqlen > 0 && scores_out) {
     const dim3 grid((s.max_seqlen + 255) / 256, s.batch);
     score_finalize_kernel<<<grid, 256, 0, stream>>>(s, cu_seqlens, cu_qlens, partial, scores_out);
     count_launches(1);
@@ -285,6 +298,13 @@ cudaError_t launch_lse_import(const Shapes& s, const float* lse_in, float* lse_w
   if (count <= 0) return cudaSuccess;
   count_launches(1);
   return launch_chained(lse_import_kernel, dim3((count + 255) / 256), dim3(256), 0, stream, count, lse_in, lse_ws);
+}
+
+cudaError_t launch_lse_export(const Shapes& s, const float* lse_ws, float* lse_out, cudaStream_t stream) {
+  const int count = s.total_q * s.hq;
+  if (count <= 0) return cudaSuccess;
+  count_launches(1);
+  return launch_chained(lse_export_kernel, dim3((count + 255) / 256), dim3(256), 0, stream, count, lse_ws, lse_out);
 }
 
 cudaError_t launch_score_generic(const Shapes& s, const Workspace& w, const void* q, const int32_t* q_idx,

@@ -350,13 +350,17 @@ cudaError_t launch_score_narrow(const Shapes& s, const Workspace& w, const void*
   const int rq = s.max_qlen;
   cudaError_t e = launch_narrow_logits(s, w, q, q_idx, cu_qlens, k, cu_seqlens, ws, device_status, stream);
   if (e != cudaSuccess) return e;
-  if (!lse_in && narrow_tail_applies(s))  // short sequences: statistics and scores in one kernel
+  if (!lse_in && scores_out && narrow_tail_applies(s))  // short sequences: statistics and scores in one kernel
     return launch_narrow_tail(s, logits, rq, scores_out, false, cu_seqlens, nullptr, nullptr, q_idx, cu_qlens, nullptr, nullptr,
                               device_status, stream);
   if (lse_in) e = launch_lse_import(s, lse_in, lse, stream);
   else e = launch_chained(score_narrow_stats_kernel, dim3(s.hq * rq, s.batch), dim3(256), 0, stream, s, cu_qlens, cu_seqlens,
                           (const float*)logits, rq, lse);
   if (e != cudaSuccess) return e;
+  if (!scores_out) {  // only the statistics were asked for (fastav_lse)
+    count_launches(lse_in ? 0 : 1);
+    return cudaGetLastError();
+  }
   if ((e = launch_chained(score_narrow_finalize_kernel, dim3((s.max_seqlen + kFinalizeThreads - 1) / kFinalizeThreads, s.batch),
                           dim3(kFinalizeThreads),
                           s.hq * rq * (sizeof(float) + sizeof(int)), stream, s, cu_qlens, cu_seqlens, (const float*)logits, rq, (const float*)lse,

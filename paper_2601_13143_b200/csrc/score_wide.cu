@@ -834,6 +834,7 @@ cudaError_t run(const Shapes& s, const Workspace& w, const CUtensorMap& k_map, c
       return e;
     count_launches(2);
   }
+  if (!scores_out) return cudaGetLastError();  // only the statistics were asked for (fastav_lse)
   if ((e = launch_chained(score_wide_kernel<DIM, 2>, dim3(grid), dim3(kThreads), smem, stream, k_map, q_map, s, q_idx, cu_qlens,
                           cu_seqlens, chunk_tiles, stat_chunks, rc_max, rows_per_chunk, (float2*)nullptr, (const float*)lse,
                           partial, (float*)nullptr, 0, device_status)) != cudaSuccess)

@@ -37,7 +37,7 @@ FASTAV_ERR_CUDA = -4
 FASTAV_ERR_TIMEOUT = -5
 
 EXPORTS = ("fastav_version", "fastav_status_string", "fastav_last_cuda_error", "fastav_workspace_bytes",
-           "fastav_score", "fastav_select", "fastav_compact", "fastav_prune", "fastav_host_arena_bytes",
+           "fastav_score", "fastav_lse", "fastav_select", "fastav_compact", "fastav_prune", "fastav_host_arena_bytes",
            "fastav_prune_host", "fastav_kernel_launches", "fastav_select_noalloc", "fastav_select_mask", "fastav_selftest_bounded_wait",
            "fastav_rollout_state_bytes", "fastav_rollout_workspace_bytes", "fastav_rollout_begin", "fastav_rollout_layer",
            "fastav_rollout_read", "fastav_rollout_threshold")
@@ -97,6 +97,8 @@ def library() -> ctypes.CDLL:
         lib.fastav_workspace_bytes.argtypes = [pp, ctypes.POINTER(ctypes.c_size_t)]
         lib.fastav_score.restype = ctypes.c_int32
         lib.fastav_score.argtypes = [pp, vp, i32p, i32p, vp, i32p, vp, vp, vp, ctypes.c_size_t, i32p, vp]
+        lib.fastav_lse.restype = ctypes.c_int32
+        lib.fastav_lse.argtypes = [pp, vp, i32p, i32p, vp, i32p, vp, vp, ctypes.c_size_t, i32p, vp]
         lib.fastav_select.restype = ctypes.c_int32
         lib.fastav_select.argtypes = [pp, vp, i32p, i32p, vp, i32p, i32p, i32p, i32p, vp, ctypes.c_size_t, i32p, vp]
         lib.fastav_compact.restype = ctypes.c_int32
@@ -199,6 +201,13 @@ def fastav_score(params, q, q_idx, cu_qlens, k, cu_seqlens, scores_out, workspac
     ws, ws_bytes = _ws(workspace)
     _check(library().fastav_score(ctypes.byref(params), _p(q), _p(q_idx), _p(cu_qlens), _p(k), _p(cu_seqlens), _p(lse_opt),
                                   _p(scores_out), ws, ws_bytes, _p(device_status), _stream(stream)), "fastav_score")
+
+
+def fastav_lse(params, q, q_idx, cu_qlens, k, cu_seqlens, lse_out, workspace, device_status=None, stream=None) -> None:
+    """Natural-log log-sum-exp of every scored row's logits per head, [total_q, Hq] (the first sweep alone)."""
+    ws, ws_bytes = _ws(workspace)
+    _check(library().fastav_lse(ctypes.byref(params), _p(q), _p(q_idx), _p(cu_qlens), _p(k), _p(cu_seqlens), _p(lse_out), ws,
+                                ws_bytes, _p(device_status), _stream(stream)), "fastav_lse")
 
 
 def fastav_select(params, scores, cu_seqlens, keep_counts, protect_opt, q_idx, cu_qlens, keep_idx_out, cu_keep_out, workspace,

@@ -97,6 +97,35 @@ def _natural_lse(p):
     return out.float()
 
 
+@pytest.mark.parametrize("lens,rows,hq,hkv,d", [([300, 40], [3, 1], 8, 2, 64), ([1000], [64], 8, 2, 128), ([777, 130, 0, 5], [40, 9, 0, 5], 28, 4, 128),
+                                                ([5000], [1], 4, 4, 64)])
+@pytest.mark.parametrize("path", ["auto", "generic", "narrow", "wide"])
+@pytest.mark.parametrize("causal", [True, False])
+def test_lse_alone_matches_float64_and_feeds_the_single_sweep_score(lens, rows, hq, hkv, d, path, causal):
+    """fastav_lse: the first sweep alone, in the attention kernels' convention; handed back as lse_opt it gives the
+    scores of the self-contained call.  |lse - ref| <= 5e-4: fp32 sums of up to a few thousand terms whose
+    exponentials are good to 1e-4 relative."""
+    if not _path_applies(path, rows, hq, hkv, d):
+        pytest.skip("path does not take these shapes")
+    p = W.random_problem(seed=17, lens=lens, rows=rows, keeps=[n // 2 for n in lens], num_q_heads=hq, num_kv_heads=hkv,
+                         head_dim=d, hidden=64, trailing_rows=False)
+    p.causal = causal
+    buf = parity.to_device(p, extra_flags=SCORE_PATHS[path])
+    lse = torch.full((p.q.shape[0], hq), float("nan"), device="cuda")
+    fastav.fastav_lse(buf.params, buf.q, buf.q_idx, buf.cu_qlens, buf.k, buf.cu_seqlens, lse, buf.workspace, buf.device_status)
+    torch.cuda.synchronize()
+    assert _sync_status(buf) == 0
+    ref = _natural_lse(p).double()
+    got = lse.cpu().double()
+    finite = torch.isfinite(ref)
+    assert torch.equal(torch.isfinite(got), finite) and (got[~finite] == float("-inf")).all()
+    assert (got[finite] - ref[finite]).abs().max() <= 5e-4 if finite.any() else True
+    fastav.fastav_score(buf.params, buf.q, buf.q_idx, buf.cu_qlens, buf.k, buf.cu_seqlens, buf.scores, buf.workspace,
+                        buf.device_status, lse_opt=lse)
+    torch.cuda.synchronize()
+    parity.assert_scores_close(buf.scores, parity.oracle_scores(p), "single sweep from fastav_lse")
+
+
 @pytest.mark.parametrize("lens,rows,hq,hkv,d", [([300, 40], [3, 1], 8, 2, 64), ([1000], [64], 8, 2, 128), ([777, 130], [40, 9], 28, 4, 128)])
 @pytest.mark.parametrize("path", ["auto", "generic"])
 def test_score_with_caller_provided_lse(lens, rows, hq, hkv, d, path):
