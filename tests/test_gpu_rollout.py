@@ -93,6 +93,25 @@ def test_rollout_with_the_attention_kernels_lse():
     _close(r_b, ref, ROLL_RTOL, "caller's statistics")
 
 
+def test_rollout_takes_the_log_sum_exp_that_fastav_lse_makes():
+    """The two calls compose: every token a scored row -> fastav_lse -> lse_opt of fastav_rollout_layer."""
+    n, hq, hkv, d, scale, alpha = 300, 8, 2, 64, 0.125, 0.6
+    qk = _layers(31, n, hq, hkv, d, 2)
+    q_idx = torch.arange(n, dtype=torch.int32, device="cuda")
+    cu = torch.tensor([0, n], dtype=torch.int32, device="cuda")
+    lse = []
+    for q, k in qk:
+        qd, kd = q.cuda(), k.cuda()
+        p = _params(n, hq, hkv, d, qd, kd, scale, True)
+        ws = torch.empty(max(fastav.fastav_workspace_bytes(p), 256), dtype=torch.uint8, device="cuda")
+        out = torch.empty(n, hq, device="cuda")
+        fastav.fastav_lse(p, qd, q_idx, cu, kd, cu, out, ws)
+        lse.append(out)
+    _, r, _ = _run(qk, n, hq, hkv, d, scale, True, alpha, lse=lse)
+    ref = orr.rollout([orr.attention_map(bf16_bits(q), bf16_bits(k), scale, True) for q, k in qk], alpha)
+    _close(r, ref, ROLL_RTOL, "rollout from fastav_lse")
+
+
 def test_rollout_limits_of_eq2():
     n, hq, hkv, d = 200, 4, 2, 64
     qk = _layers(9, n, hq, hkv, d, 2)
