@@ -26,6 +26,19 @@ def test_eq3_multiplies_the_newest_layer_from_the_left():
     assert np.allclose(orr.rollout([a1, a2], 0.5), [[13 / 16, 3 / 16], [0.25, 0.75]], atol=0, rtol=1e-15)
 
 
+def test_hand_worked_fixture(golden_dir):
+    import json
+    import os
+    with open(os.path.join(golden_dir, "eq23_hand_worked.json")) as f:
+        cases = json.load(f)["cases"]
+    assert len(cases) >= 3
+    for c in cases:
+        r = orr.rollout([np.array(m) for m in c["maps"]], c["alpha"])
+        assert np.allclose(r, np.array(c["rollout"]), rtol=1e-14, atol=0), c["name"]
+        if "importance" in c:
+            assert np.allclose(orr.importance(r), c["importance"], rtol=1e-14), c["name"]
+
+
 def test_eq2_limits():
     rng = np.random.default_rng(0)
     a = rng.random((5, 5))
