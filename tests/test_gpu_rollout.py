@@ -181,6 +181,21 @@ def test_rollout_at_the_papers_prompt_size():
     assert r[0, 0] == 1.0
 
 
+def test_rollout_of_a_long_sequence_on_sampled_rows():
+    """6,000 tokens (47 tiles a side, ragged last tile): rows of R sampled across the sequence against the oracle
+    (row i of A~2 A~1 needs only row i of A~2), plus what holds for every row."""
+    n, hq, hkv, d, alpha, scale = 6000, 4, 2, 64, 0.5, 0.125
+    qk = _layers(6, n, hq, hkv, d, 2)
+    imp, r, _ = _run(qk, n, hq, hkv, d, scale, True, alpha)
+    a1 = orr.with_residual(orr.attention_map(bf16_bits(qk[0][0]), bf16_bits(qk[0][1]), scale, True), alpha)
+    a2 = orr.with_residual(orr.attention_map(bf16_bits(qk[1][0]), bf16_bits(qk[1][1]), scale, True), alpha)
+    rows = [0, 1, 127, 128, 129, 2999, 4095, 4096, 5887, 5888, 5998, 5999]
+    _close(r[rows], a2[rows] @ a1, ROLL_RTOL, "sampled rows")
+    assert np.allclose(r.sum(axis=1), 1.0, atol=2e-4)
+    assert np.array_equal(np.triu(r, 1), np.zeros_like(r))
+    assert abs(imp.sum() - 1.0) < 2e-4
+
+
 def test_rollout_argument_errors():
     n, hq, hkv, d = 64, 4, 2, 64
     q, k = [t.cuda() for t in _layers(1, n, hq, hkv, d, 1)[0]]
