@@ -209,17 +209,19 @@ __global__ void __launch_bounds__(256) score_narrow_stats_kernel(Shapes s, const
   if (r >= rows) return;
   const float* z = logits + ((long long)head * rq + r) * s.total_tokens + tok0;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  // One pass: every thread keeps a running (max, sum 2^(z - max)) over its strided share, four loads at a time.
+  // One pass: every thread keeps a running (max, sum 2^(z - max)) over its strided share, sixteen loads at a time.
   float m = -INFINITY, l = 0.f;
-  for (int j0 = threadIdx.x; j0 < n; j0 += 256 * 4) {
-    float v[4];
+  for (int j0 = threadIdx.x; j0 < n; j0 += 256 * 16) {  // sixteen loads in flight per thread: two trips for 8k tokens
+    float v[16];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) v[u] = j0 + u * 256 < n ? chain_load(z + j0 + u * 256) : -INFINITY;
-    const float m_new = fmaxf(fmaxf(m, fmaxf(v[0], v[1])), fmaxf(v[2], v[3]));
+    for (int u = 0; u < 16; ++u) v[u] = j0 + u * 256 < n ? chain_load(z + j0 + u * 256) : -INFINITY;
+    float m_new = m;
+#pragma unroll
+    for (int u = 0; u < 16; ++u) m_new = fmaxf(m_new, v[u]);
     if (m_new > -INFINITY) {
       l = l * exp2f(m - m_new);
 #pragma unroll
-      for (int u = 0; u < 4; ++u) l += exp2f(v[u] - m_new);
+      for (int u = 0; u < 16; ++u) l += exp2f(v[u] - m_new);
       m = m_new;
     }
   }
