@@ -254,8 +254,7 @@ def attention_lse(p, buf) -> torch.Tensor:
 
 def oracle_sample(w: W.Workload):
     """Bounded sample for the CPU legs: the first sequence of every stage."""
-    sys.path.insert(0, os.path.join(ROOT, "tests"))
-    from conftest import bf16_bits
+    bf16_bits = W.bf16_bits
     sample = []
     for si in range(len(w.stages)):
         p = W.make_stage(w, si)

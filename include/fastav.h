@@ -8,7 +8,7 @@
  * the middle layer and the "fine" stage at every later layer.  This library is that step:
  *
  *     fastav_score    Eq. 4, generalised to R scored rows, grouped-query heads, varlen batches
- *     fastav_select   "tokens with the lowest P% scores are removed": top-k keep set
+ *     fastav_select   the bottom-P % rule of Section 2.2 as a top-k keep set
  *     fastav_compact  the survivor layout: gather hidden states, position ids, K and V rows
  *     fastav_prune    all three in one enqueue
  *
@@ -79,11 +79,16 @@ extern "C" {
 #define FASTAV_DEV_PROTECT_OVERFLOW 2 /* more protected tokens than k_b: the lowest-index ones were kept */
 #define FASTAV_DEV_WAIT_EXPIRED 4     /* a bounded wait inside a kernel ran out; results of that call are invalid */
 #define FASTAV_DEV_BAD_INDEX 8        /* fastav_compact met a keep_idx entry outside its sequence and skipped that row */
+#define FASTAV_DEV_SHAPE_MISMATCH 16  /* cu_seqlens / cu_qlens on the device disagree with the host scalars of params (a sequence
+                                         longer than max_seqlen, a batch longer than total_tokens, more scored rows than max_qlen /
+                                         total_q, more work than the launch was sized for): the excess was left out */
+#define FASTAV_DEV_SLOW_PATH 32       /* informational: fastav_score could not describe q or k to the tensor-memory-accelerator
+                                         (tensor-map encoding refused) and ran its CUDA-core tiles instead, much more slowly */
 
 /*
  * Shapes of one prune call (host memory).  The counts that fix grid sizes and output sizes are
  * host scalars because the caller knows them without a device round trip: k_b is a function of
- * n_b ("lowest P%" -> k_b = n_b - floor(P n_b)).
+ * n_b (bottom P % removed -> k_b = n_b - floor(P n_b)).
  */
 typedef struct fastav_params {
   int32_t batch;                    /* B >= 1 */
@@ -160,7 +165,7 @@ int32_t fastav_lse(const fastav_params* params, const void* q, const int32_t* q_
                    void* stream);
 
 /*
- * "Tokens with the lowest P% scores are removed" (Section 2.2): per sequence keep the
+ * The bottom-P % rule of Section 2.2 ("Fine pruning"), stated on the survivors: per sequence keep the
  * keep_counts[b] highest-scoring tokens; equal scores go to the lower index; protected tokens
  * (protect_opt[j] != 0, and the scored rows' tokens under FASTAV_PROTECT_QUERY_ROWS) rank above
  * every score.  Survivors are written in ascending index order.
@@ -198,7 +203,7 @@ int32_t fastav_select_mask(const fastav_params* params, const uint8_t* keep_mask
                            int32_t* device_status, void* stream);
 
 /*
- * Survivor layout (what "iteratively refining the token set" in Section 2.2 leaves for the next
+ * Survivor layout (what the layer-by-layer shrinking of the token set in Section 2.2 leaves for the next
  * layer): output row cu_keep[b] + i is input row cu_seqlens[b] + keep_idx[cu_keep[b] + i] of
  *
  *   hidden  [N, hidden] bf16   -> hidden_out [total_keep, hidden]
@@ -216,10 +221,14 @@ int32_t fastav_compact(const fastav_params* params, const int32_t* keep_idx, con
 /*
  * The whole prune step of one pruning layer (Fig. 3; Section 2.2): fastav_score, fastav_select
  * and fastav_compact enqueued back to back.  scores_out, keep_idx_out and cu_keep_out are still
- * written, so the caller can inspect or reuse them.  Arguments as in the three calls above.
+ * written, so the caller can inspect or reuse them.  The argument list is the union of the three
+ * calls above, each argument with the meaning it has there -- lse_opt included: a caller whose
+ * attention kernel already returned the log-sum-exp of the scored rows for this layer (Section 1:
+ * the method works beside FlashAttention-style kernels) passes it and the scores take one sweep
+ * over K; NULL makes the call self-contained.
  */
 int32_t fastav_prune(const fastav_params* params, const void* q, const int32_t* q_idx, const int32_t* cu_qlens,
-                     const void* k, const void* v, const int32_t* cu_seqlens, const int32_t* keep_counts,
+                     const void* k, const void* v, const int32_t* cu_seqlens, const float* lse_opt, const int32_t* keep_counts,
                      const uint8_t* protect_opt, const void* hidden_in, const int32_t* pos_in, float* scores_out,
                      int32_t* keep_idx_out, int32_t* cu_keep_out, void* hidden_out, int32_t* pos_out, void* k_out,
                      void* v_out, void* workspace, size_t workspace_bytes, int32_t* device_status, void* stream);
@@ -232,12 +241,14 @@ int32_t fastav_prune(const fastav_params* params, const void* q, const int32_t* 
  * optional) on `stream`, staged through `device_arena`, a DEVICE buffer of at least
  * fastav_host_arena_bytes() bytes, 256-byte aligned, owned by the caller.  Host outputs are valid
  * once the stream has been synchronised.  Only packed layouts are accepted (token stride =
- * heads * head_dim, head stride = head_dim; otherwise FASTAV_ERR_UNSUPPORTED).  The paper has no
+ * heads * head_dim, head stride = head_dim; otherwise FASTAV_ERR_UNSUPPORTED).  Every check of
+ * fastav_prune is made before the first copy, so a negative return value leaves nothing enqueued.
+ * FASTAV_CHAIN_CALLS is ignored: the index arrays are uploaded by this very call.  The paper has no
  * counterpart for this entry point; it computes exactly what fastav_prune computes.
  */
 int32_t fastav_host_arena_bytes(const fastav_params* params, size_t* out_bytes);
 int32_t fastav_prune_host(const fastav_params* params, const void* q, const int32_t* q_idx, const int32_t* cu_qlens,
-                          const void* k, const void* v, const int32_t* cu_seqlens, const int32_t* keep_counts,
+                          const void* k, const void* v, const int32_t* cu_seqlens, const float* lse_opt, const int32_t* keep_counts,
                           const uint8_t* protect_opt, const void* hidden_in, const int32_t* pos_in, float* scores_out,
                           int32_t* keep_idx_out, int32_t* cu_keep_out, void* hidden_out, int32_t* pos_out, void* k_out,
                           void* v_out, int32_t* status_out, void* device_arena, size_t arena_bytes, void* stream);
@@ -310,8 +321,8 @@ int32_t fastav_selftest_bounded_wait(int32_t limit_ms, int32_t* device_status, v
  *                          Of params: batch (must be 1), total_tokens = total_q = max_seqlen = max_qlen = n,
  *                          head counts, head_dim (64 or 128), q/k strides, softmax_scale, FASTAV_CAUSAL.
  *                          Workspace: 256-byte aligned, fastav_rollout_workspace_bytes(params) bytes.
- *   fastav_rollout_read    importance_out [n] fp32: mean over rows of column j of R, "how much each token
- *                          from the input layer influences every other token"; rollout_out_opt: NULL or
+ *   fastav_rollout_read    importance_out [n] fp32: mean over rows of column j of R (Section 2.1 after Eq. 3:
+ *                          the influence of input token j on all tokens); rollout_out_opt: NULL or
  *                          [n, n] fp32 row-major R.  `layers_applied` = number of fastav_rollout_layer calls.
  *   fastav_rollout_threshold  keep_mask_out [n] uint8 = importance[j] >= threshold, or protect_opt[j] != 0;
  *                          *cut_out (device int32) = one past the last unprotected token that reaches the

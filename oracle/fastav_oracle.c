@@ -15,8 +15,8 @@
  * generalised to R scored query rows instead
  * of one (mean over rows and heads), grouped-query attention (query head h
  * reads KV head h / G), an optional causal mask by token index, an explicit
- * softmax scale, and variable-length batches.  Then "tokens with the lowest P%
- * scores are removed" (same paragraph): keep the k largest, ties to the lower
+ * softmax scale, and variable-length batches.  Then the bottom-P % rule of the
+ * same paragraph, stated on the survivors: keep the k largest, ties to the lower
  * index, protected tokens always kept; survivors stay in their original order
  * and carry their rows of hidden states, position ids, K and V with them.
  *
@@ -163,7 +163,7 @@ static int ascending_i32(const void *pa, const void *pb) {
 }
 
 /*
- * "Tokens with the lowest P% scores are removed": per sequence keep the k_b
+ * The bottom-P % rule (Section 2.2, "Fine pruning"): per sequence keep the k_b
  * tokens that come first when tokens are ranked by (score descending, index
  * ascending); protected tokens rank as +infinity.  The decision is taken on
  * fp32 scores, the precision the CUDA selector works in.  k_b is clamped to

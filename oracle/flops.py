@@ -21,7 +21,7 @@ def layer_flops(n: int, hidden: int, ffn: int) -> int:
 
 
 def removed_count(n: int, prune_ratio: float) -> int:
-    """Tokens removed when "the lowest P%" of n tokens go: floor(P n)."""
+    """Tokens removed by the bottom-P % rule (Section 2.2, "Fine pruning") from n tokens: floor(P n)."""
     return int(math.floor(prune_ratio * n + 1e-6))
 
 
@@ -43,7 +43,7 @@ def relative_flops(n0: int, num_layers: int, hidden: int, ffn: int, prunes: dict
 
 
 def fastav_schedule(n0: int, num_layers: int, global_layer: int, global_keep: int, fine_ratio: float) -> dict[int, int]:
-    """The paper's two-stage schedule: a global prune at the middle layer, then "the lowest P%"
+    """The paper's two-stage schedule: a global prune at the middle layer, then the bottom P %
     removed at every following layer (Section 2.2; P = 20% in Section 3.1)."""
     prunes = {global_layer: global_keep}
     n = global_keep

@@ -9,8 +9,8 @@ token importance via attention rollout", Eq. 2 and Eq. 3).  Nothing here is shar
 
 Readings where the paper is silent: the attention weights are the model's own (softmax of scale * q.k over
 the keys a row may see, causal by index, query head h reading KV head h // G); alpha is a parameter; the
-importance of input token j is the mean over rows of column j of R ("how much each token from the input
-layer influences every other token"); the threshold keeps the tokens whose importance reaches it, and the
+importance of input token j is the mean over rows of column j of R (Section 2.1 after Eq. 3: the influence of
+each input-layer token on all tokens); the threshold keeps the tokens whose importance reaches it, and the
 positional rule the paper derives from it is "keep everything before the last such token".
 """
 from __future__ import annotations

@@ -34,13 +34,13 @@ int32_t check_params(const fastav_params* p) {
 
 // A [tokens, heads, dim] view: the head stride must hold a row, the token stride must hold all heads,
 // and both must keep rows 16-byte aligned.
+// Two layouts pass: heads inside a token (st >= heads * sh, e.g. a view into a packed projection output) and
+// tokens inside a head (sh > st, a head-major cache; its extent is the caller's business).  What is rejected is
+// the one case that is certainly wrong: heads inside a token whose rows overlap the next token's.
 int32_t check_strides(int64_t st, int64_t sh, int heads, int dim) {
   if (sh < dim || st < dim) return FASTAV_ERR_INVALID_ARG;
-  if (heads > 1 && st < sh && sh < (int64_t)dim * heads) {
-    // head-major inside a token needs st >= heads*sh; token-major inside a head needs sh >= tokens*st,
-    // which cannot be checked without the extent: accept only the first form when st >= sh.
-  }
   if (st % 8 != 0 || sh % 8 != 0) return FASTAV_ERR_UNSUPPORTED;
+  if (heads > 1 && st >= sh && st < (int64_t)(heads - 1) * sh + dim) return FASTAV_ERR_INVALID_ARG;
   return FASTAV_OK;
 }
 
@@ -150,6 +150,12 @@ Workspace plan_workspace(const fastav_params& p) {
   return w;
 }
 
+__global__ void status_or_kernel(int32_t* device_status, int32_t bits) {
+  pdl_trigger();
+  pdl_wait();
+  atomicOr(device_status, bits);
+}
+
 // A forced score path (FASTAV_SCORE_PATH_*) must support the shapes; the shape-based choice always does.
 bool score_path_ok(const Shapes& s) {
   const unsigned forced = s.flags & FASTAV_SCORE_PATH_MASK;
@@ -172,8 +178,33 @@ cudaError_t launch_score(const Shapes& s, const Workspace& w, const void* q, con
     const cudaError_t e = launch_score_wide(s, w, q, q_idx, cu_qlens, k, cu_seqlens, lse_in, scores_out, ws, device_status, stream, &used);
     if (used || e != cudaSuccess) return e;
     if (forced == FASTAV_SCORE_PATH_WIDE) return cudaErrorNotSupported;
+    // The tensor map could not be encoded: the CUDA-core tiles below are correct but far slower, so say so.
+    if (device_status) {
+      const cudaError_t es = launch_chained(status_or_kernel, dim3(1), dim3(1), 0, stream, device_status, (int32_t)FASTAV_DEV_SLOW_PATH);
+      if (es != cudaSuccess) return es;
+      count_launches(1);
+    }
   }
   return launch_score_generic(s, w, q, q_idx, cu_qlens, k, cu_seqlens, lse_in, scores_out, ws, stream);
+}
+
+// Everything fastav_prune checks before it enqueues anything (also used by the host-buffer entry point, which must
+// not start its uploads for a call that will be refused).
+int32_t validate_prune(const fastav_params* params, const void* q, const int32_t* q_idx, const int32_t* cu_qlens, const void* k,
+                       const void* v, const int32_t* cu_seqlens, const int32_t* keep_counts, const void* hidden_in,
+                       const int32_t* pos_in, const float* scores_out, const int32_t* keep_idx_out, const int32_t* cu_keep_out,
+                       const void* hidden_out, const int32_t* pos_out, const void* k_out, const void* v_out, const void* workspace,
+                       size_t workspace_bytes) {
+  int32_t rc = check_params(params);
+  if (rc != FASTAV_OK) return rc;
+  if ((rc = check_score_args(params, q, q_idx, cu_qlens, k, cu_seqlens, scores_out)) != FASTAV_OK) return rc;
+  if ((rc = check_select_args(params, scores_out, cu_seqlens, keep_counts, q_idx, cu_qlens, keep_idx_out, cu_keep_out)) != FASTAV_OK) return rc;
+  if ((rc = check_compact_args(params, keep_idx_out, cu_keep_out, cu_seqlens, hidden_in, hidden_out, pos_in, pos_out, k, k_out,
+                               v, v_out)) != FASTAV_OK)
+    return rc;
+  if ((rc = check_workspace(plan_workspace(*params), workspace, workspace_bytes)) != FASTAV_OK) return rc;
+  if (!score_path_ok(make_shapes(*params))) return FASTAV_ERR_UNSUPPORTED;
+  return FASTAV_OK;
 }
 
 }  // namespace fastav
@@ -277,35 +308,30 @@ int32_t fastav_compact(const fastav_params* params, const int32_t* keep_idx, con
 }
 
 int32_t fastav_prune(const fastav_params* params, const void* q, const int32_t* q_idx, const int32_t* cu_qlens,
-                     const void* k, const void* v, const int32_t* cu_seqlens, const int32_t* keep_counts,
+                     const void* k, const void* v, const int32_t* cu_seqlens, const float* lse_opt, const int32_t* keep_counts,
                      const uint8_t* protect_opt, const void* hidden_in, const int32_t* pos_in, float* scores_out,
                      int32_t* keep_idx_out, int32_t* cu_keep_out, void* hidden_out, int32_t* pos_out, void* k_out,
                      void* v_out, void* workspace, size_t workspace_bytes, int32_t* device_status, void* stream) {
   // Validate everything first so that an error leaves nothing enqueued.
-  int32_t rc = check_params(params);
+  int32_t rc = validate_prune(params, q, q_idx, cu_qlens, k, v, cu_seqlens, keep_counts, hidden_in, pos_in, scores_out, keep_idx_out,
+                              cu_keep_out, hidden_out, pos_out, k_out, v_out, workspace, workspace_bytes);
   if (rc != FASTAV_OK) return rc;
   chain_begin(params->flags);
-  if ((rc = check_score_args(params, q, q_idx, cu_qlens, k, cu_seqlens, scores_out)) != FASTAV_OK) return rc;
-  if ((rc = check_select_args(params, scores_out, cu_seqlens, keep_counts, q_idx, cu_qlens, keep_idx_out, cu_keep_out)) != FASTAV_OK) return rc;
-  if ((rc = check_compact_args(params, keep_idx_out, cu_keep_out, cu_seqlens, hidden_in, hidden_out, pos_in, pos_out, k, k_out,
-                               v, v_out)) != FASTAV_OK)
-    return rc;
   const Workspace w = plan_workspace(*params);
-  if ((rc = check_workspace(w, workspace, workspace_bytes)) != FASTAV_OK) return rc;
   const Shapes s = make_shapes(*params);
-  if (!score_path_ok(s)) return FASTAV_ERR_UNSUPPORTED;
   unsigned char* ws = static_cast<unsigned char*>(workspace);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e = cudaSuccess;
   const unsigned forced = s.flags & FASTAV_SCORE_PATH_MASK;
-  if (params->total_tokens > 0 && score_narrow_applies(s) && narrow_tail_applies(s) && (forced == 0 || forced == FASTAV_SCORE_PATH_NARROW)) {
+  if (params->total_tokens > 0 && !lse_opt && score_narrow_applies(s) && narrow_tail_applies(s) &&
+      (forced == 0 || forced == FASTAV_SCORE_PATH_NARROW)) {
     // Short sequences, few scored rows: logits, then ONE kernel for the softmax statistics, the scores and the keep list.
     e = launch_narrow_logits(s, w, q, q_idx, cu_qlens, k, cu_seqlens, ws, device_status, st);
     if (e == cudaSuccess)
       e = launch_narrow_tail(s, reinterpret_cast<const float*>(ws + w.logits_off), s.max_qlen, scores_out, true, cu_seqlens,
                              keep_counts, protect_opt, q_idx, cu_qlens, keep_idx_out, cu_keep_out, device_status, st);
   } else {
-    if (params->total_tokens > 0) e = launch_score(s, w, q, q_idx, cu_qlens, k, cu_seqlens, nullptr, scores_out, ws, device_status, st);
+    if (params->total_tokens > 0) e = launch_score(s, w, q, q_idx, cu_qlens, k, cu_seqlens, lse_opt, scores_out, ws, device_status, st);
     if (e == cudaSuccess)
       e = launch_select(s, w, scores_out, cu_seqlens, keep_counts, protect_opt, q_idx, cu_qlens, keep_idx_out, cu_keep_out, ws,
                         device_status, st);

@@ -95,6 +95,12 @@ cudaError_t launch_compact(const Shapes& s, const int32_t* keep_idx, const int32
                            int32_t* pos_out, const void* k_in, void* k_out, const void* v_in, void* v_out,
                            int32_t* device_status, cudaStream_t stream);
 
+int32_t validate_prune(const fastav_params* params, const void* q, const int32_t* q_idx, const int32_t* cu_qlens, const void* k,
+                       const void* v, const int32_t* cu_seqlens, const int32_t* keep_counts, const void* hidden_in,
+                       const int32_t* pos_in, const float* scores_out, const int32_t* keep_idx_out, const int32_t* cu_keep_out,
+                       const void* hidden_out, const int32_t* pos_out, const void* k_out, const void* v_out, const void* workspace,
+                       size_t workspace_bytes);
+
 // Diagnostic launch counter (fastav_kernel_launches).
 void count_launches(int n);
 
@@ -112,6 +118,32 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a -
 // global memory another kernel may still read.  Every block waits before it exits, so completion of a
 // kernel implies completion of all its predecessors.
 #ifdef __CUDACC__
+// Sequence b of a packed batch as the device sees it in a prefix-sum array, cut down to what the host scalars
+// promise: buffers and grids are sized from total_tokens / max_seqlen (total_q / max_qlen), loop bounds come from
+// the device array, and a caller whose two views disagree must get a status bit, not an out-of-bounds access.
+struct Span {
+  int first, count;
+  bool bad;  // the array and the host scalars disagree: the span was clamped (FASTAV_DEV_SHAPE_MISMATCH)
+};
+__device__ __forceinline__ Span checked_span(const int32_t* cu, int b, int total, int max_count) {
+  const int a = cu[b], e = cu[b + 1];
+  Span sp{a, e - a, false};
+  if (a < 0 || a > total) {
+    sp = Span{0, 0, true};
+  } else {
+    const int room = min(max_count, total - a);
+    if (sp.count < 0) { sp.count = 0; sp.bad = true; }
+    else if (sp.count > room) { sp.count = room; sp.bad = true; }
+  }
+  return sp;
+}
+__device__ __forceinline__ Span seq_span(const Shapes& s, const int32_t* cu_seqlens, int b) {
+  return checked_span(cu_seqlens, b, s.total_tokens, s.max_seqlen);
+}
+__device__ __forceinline__ Span row_span(const Shapes& s, const int32_t* cu_qlens, int b) {
+  return checked_span(cu_qlens, b, s.total_q, s.max_qlen);
+}
+
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 // A pointer to data the predecessor writes must be passed through this after pdl_wait: the compiler

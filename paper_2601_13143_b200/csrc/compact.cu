@@ -1,6 +1,6 @@
 // Survivor gather: out[i] = in[source(i)] for hidden states, K, V and position ids.
 //
-// The step the paper implies by "iteratively refining the token set" (Section 2.2): the following
+// The step Section 2.2 ("Fine pruning") implies when it shrinks the token set layer after layer: the following
 // layers only ever see the survivors, so their rows are packed into a dense layout.  It moves
 // about 85-90 % of all bytes of a prune call and is bound by HBM bandwidth: each row (7-8 KB of
 // hidden state, 1-2 KB each of K and V) is read once and written once with 16-byte accesses, the
@@ -22,7 +22,8 @@ constexpr int kUnroll = 4;  // 16-byte loads in flight per thread
 
 __device__ __forceinline__ uint4 load_stream(const uint4* p) {
   uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+  // a plain (coherent) load: under programmatic launch the rows may be what the previous kernel wrote
+  asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                : "l"(p));
   return v;

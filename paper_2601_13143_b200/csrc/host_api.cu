@@ -9,7 +9,7 @@ namespace fastav {
 namespace {
 
 struct Arena {
-  size_t q, q_idx, cu_qlens, k, v, cu_seqlens, keep_counts, protect, hidden, pos;
+  size_t q, q_idx, cu_qlens, k, v, cu_seqlens, lse, keep_counts, protect, hidden, pos;
   size_t scores, keep_idx, cu_keep, hidden_out, pos_out, k_out, v_out, status, workspace, workspace_bytes, total;
 };
 
@@ -33,6 +33,7 @@ Arena plan_arena(const fastav_params& p) {
   a.k = carve(N * kv_row);
   a.v = carve(N * kv_row);
   a.cu_seqlens = carve((B + 1) * 4);
+  a.lse = carve(R * p.num_q_heads * 4);
   a.keep_counts = carve(B * 4);
   a.protect = carve(N);
   a.hidden = carve(N * (size_t)p.hidden * 2);
@@ -69,10 +70,10 @@ int32_t fastav_host_arena_bytes(const fastav_params* params, size_t* out_bytes) 
 }
 
 int32_t fastav_prune_host(const fastav_params* params, const void* q, const int32_t* q_idx, const int32_t* cu_qlens,
-                          const void* k, const void* v, const int32_t* cu_seqlens, const int32_t* keep_counts,
-                          const uint8_t* protect_opt, const void* hidden_in, const int32_t* pos_in, float* scores_out,
-                          int32_t* keep_idx_out, int32_t* cu_keep_out, void* hidden_out, int32_t* pos_out, void* k_out,
-                          void* v_out, int32_t* status_out, void* device_arena, size_t arena_bytes, void* stream) {
+                          const void* k, const void* v, const int32_t* cu_seqlens, const float* lse_opt,
+                          const int32_t* keep_counts, const uint8_t* protect_opt, const void* hidden_in, const int32_t* pos_in,
+                          float* scores_out, int32_t* keep_idx_out, int32_t* cu_keep_out, void* hidden_out, int32_t* pos_out,
+                          void* k_out, void* v_out, int32_t* status_out, void* device_arena, size_t arena_bytes, void* stream) {
   size_t need = 0;
   int32_t rc = fastav_host_arena_bytes(params, &need);
   if (rc != FASTAV_OK) return rc;
@@ -82,12 +83,23 @@ int32_t fastav_prune_host(const fastav_params* params, const void* q, const int3
   if ((v == nullptr) != (v_out == nullptr) || (hidden_in == nullptr) != (hidden_out == nullptr) ||
       (pos_in == nullptr) != (pos_out == nullptr) || !k_out)
     return FASTAV_ERR_INVALID_ARG;
-  const fastav_params& p = *params;
+  // The index arrays are uploaded by this very call, so its first kernel must not start before earlier work on
+  // the stream has completed: the chaining flag is not forwarded.
+  fastav_params p = *params;
+  p.flags &= ~FASTAV_CHAIN_CALLS;
   const Arena a = plan_arena(p);
   unsigned char* base = static_cast<unsigned char*>(device_arena);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t N = p.total_tokens, K = p.total_keep, B = p.batch, R = p.total_q;
   const size_t kv_row = (size_t)p.num_kv_heads * p.head_dim * 2;
+  auto dev = [&](size_t off, const void* host) -> void* { return host ? base + off : nullptr; };
+  // Everything the fused call would refuse is refused here, before the first copy is enqueued.
+  rc = validate_prune(&p, base + a.q, (const int32_t*)(base + a.q_idx), (const int32_t*)(base + a.cu_qlens), base + a.k, dev(a.v, v),
+                      (const int32_t*)(base + a.cu_seqlens), (const int32_t*)(base + a.keep_counts), dev(a.hidden, hidden_in),
+                      (const int32_t*)dev(a.pos, pos_in), (const float*)(base + a.scores), (const int32_t*)(base + a.keep_idx),
+                      (const int32_t*)(base + a.cu_keep), dev(a.hidden_out, hidden_out), (const int32_t*)dev(a.pos_out, pos_out),
+                      base + a.k_out, dev(a.v_out, v_out), base + a.workspace, a.workspace_bytes);
+  if (rc != FASTAV_OK) return rc;
   cudaError_t e = cudaSuccess;
   auto h2d = [&](size_t off, const void* src, size_t bytes) {
     if (e == cudaSuccess && src && bytes) e = cudaMemcpyAsync(base + off, src, bytes, cudaMemcpyHostToDevice, st);
@@ -101,15 +113,16 @@ int32_t fastav_prune_host(const fastav_params* params, const void* q, const int3
   h2d(a.k, k, N * kv_row);
   h2d(a.v, v, N * kv_row);
   h2d(a.cu_seqlens, cu_seqlens, (B + 1) * 4);
+  h2d(a.lse, lse_opt, R * p.num_q_heads * 4);
   h2d(a.keep_counts, keep_counts, B * 4);
   h2d(a.protect, protect_opt, N);
   h2d(a.hidden, hidden_in, N * (size_t)p.hidden * 2);
   h2d(a.pos, pos_in, N * 4);
   if (e == cudaSuccess) e = cudaMemsetAsync(base + a.status, 0, 4, st);
   if (e != cudaSuccess) return FASTAV_ERR_CUDA;
-  auto dev = [&](size_t off, const void* host) -> void* { return host ? base + off : nullptr; };
-  rc = fastav_prune(params, base + a.q, (const int32_t*)(base + a.q_idx), (const int32_t*)(base + a.cu_qlens), base + a.k,
-                    dev(a.v, v), (const int32_t*)(base + a.cu_seqlens), (const int32_t*)(base + a.keep_counts),
+  rc = fastav_prune(&p, base + a.q, (const int32_t*)(base + a.q_idx), (const int32_t*)(base + a.cu_qlens), base + a.k,
+                    dev(a.v, v), (const int32_t*)(base + a.cu_seqlens), (const float*)dev(a.lse, lse_opt),
+                    (const int32_t*)(base + a.keep_counts),
                     (const uint8_t*)dev(a.protect, protect_opt), dev(a.hidden, hidden_in), (const int32_t*)dev(a.pos, pos_in),
                     (float*)(base + a.scores), (int32_t*)(base + a.keep_idx), (int32_t*)(base + a.cu_keep),
                     dev(a.hidden_out, hidden_out), (int32_t*)dev(a.pos_out, pos_out), base + a.k_out, dev(a.v_out, v_out),

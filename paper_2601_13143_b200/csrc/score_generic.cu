@@ -88,8 +88,9 @@ template <int DIM>
 __device__ __forceinline__ bool load_key_tile(TileShared<DIM>& sh, const Shapes& s, const uint16_t* k,
                                               const int32_t* cu_seqlens, int& tok0, int& n, int& key0, int& keys_valid) {
   const int b = blockIdx.z, g = blockIdx.y;
-  tok0 = cu_seqlens[b];
-  n = cu_seqlens[b + 1] - tok0;
+  const Span seq = seq_span(s, cu_seqlens, b);
+  tok0 = seq.first;
+  n = seq.count;
   key0 = blockIdx.x * kTileKeys;
   if (key0 >= n) return false;
   keys_valid = min(kTileKeys, n - key0);
@@ -121,7 +122,9 @@ __global__ void __launch_bounds__(kThreads) score_tile_stats_kernel(Shapes s, co
   TileShared<DIM>& sh = *reinterpret_cast<TileShared<DIM>*>(smem_raw);
   int tok0, n, key0, keys_valid;
   if (!load_key_tile<DIM>(sh, s, k, cu_seqlens, tok0, n, key0, keys_valid)) return;
-  const int b = blockIdx.z, row0 = cu_qlens[b], rows = cu_qlens[b + 1] - row0;
+  const int b = blockIdx.z;
+  const Span qrows = row_span(s, cu_qlens, b);
+  const int row0 = qrows.first, rows = qrows.count;
   const int flat_count = rows * s.group;
   const bool causal = (s.flags & FASTAV_CAUSAL) != 0;
   for (int flat0 = 0; flat0 < flat_count; flat0 += kTileRows) {
@@ -165,7 +168,7 @@ __global__ void __launch_bounds__(256) score_merge_stats_kernel(Shapes s, const 
     const int mid = (lo + hi) >> 1;
     if (cu_qlens[mid] <= row) lo = mid; else hi = mid;
   }
-  const int n = cu_seqlens[lo + 1] - cu_seqlens[lo];
+  const int n = seq_span(s, cu_seqlens, lo).count;
   const int tiles = (n + kTileKeys - 1) / kTileKeys;
   const float2* mine = stats + (long long)warp * stat_tiles;
   float m = -INFINITY;
@@ -195,7 +198,9 @@ __global__ void __launch_bounds__(kThreads) score_tile_accumulate_kernel(Shapes 
   TileShared<DIM>& sh = *reinterpret_cast<TileShared<DIM>*>(smem_raw);
   int tok0, n, key0, keys_valid;
   if (!load_key_tile<DIM>(sh, s, k, cu_seqlens, tok0, n, key0, keys_valid)) return;
-  const int b = blockIdx.z, row0 = cu_qlens[b], rows = cu_qlens[b + 1] - row0;
+  const int b = blockIdx.z;
+  const Span qrows = row_span(s, cu_qlens, b);
+  const int row0 = qrows.first, rows = qrows.count;
   const int flat_count = rows * s.group;
   const bool causal = (s.flags & FASTAV_CAUSAL) != 0;
   // 4 threads per key, 8 rows of the chunk each.
@@ -226,8 +231,9 @@ __global__ void __launch_bounds__(256) score_finalize_kernel(Shapes s, const int
                                                              const int32_t* __restrict__ cu_qlens,
                                                              const float* __restrict__ partial, float* __restrict__ scores) {
   const int b = blockIdx.y;
-  const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
-  const int rows = cu_qlens[b + 1] - cu_qlens[b];
+  const Span seq = seq_span(s, cu_seqlens, b);
+  const int tok0 = seq.first, n = seq.count;
+  const int rows = row_span(s, cu_qlens, b).count;
   const float inv = rows > 0 ? 1.0f / ((float)s.hq * (float)rows) : 0.f;
   for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < n; j += gridDim.x * blockDim.x) {
     float total = 0.f;

@@ -72,11 +72,13 @@ score_narrow_logits_kernel(Shapes s, const uint16_t* __restrict__ q, const int32
   pdl_acquire(q);
   pdl_acquire(k);
   const int b = blockIdx.z;
-  const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
+  const Span seq = seq_span(s, cu_seqlens, b), qrows = row_span(s, cu_qlens, b);
+  if ((seq.bad || qrows.bad) && threadIdx.x == 0 && device_status) atomicOr(device_status, FASTAV_DEV_SHAPE_MISMATCH);
+  const int tok0 = seq.first, n = seq.count;
   const int key_begin = blockIdx.x * chunk_keys;
   if (key_begin >= n) return;
   const int key_end = min(n, key_begin + chunk_keys);
-  const int row0 = cu_qlens[b], rows = min(cu_qlens[b + 1] - row0, rq);
+  const int row0 = qrows.first, rows = min(qrows.count, rq);
   const int flat_rows = rows * s.group;
   if (flat_rows == 0) return;
   const int passes = (flat_rows + ROWS - 1) / ROWS;
@@ -142,7 +144,11 @@ score_narrow_logits_kernel(Shapes s, const uint16_t* __restrict__ q, const int32
 
     for (int sl = 0; sl < slots; ++sl, ++it) {
       const int stage = it % kStages;
-      if (!ptx::mbar_wait_bounded(ptx::smem_u32(&full[stage]), (it / kStages) & 1, &abort_flag)) return;
+      if (!ptx::mbar_wait_bounded(ptx::smem_u32(&full[stage]), (it / kStages) & 1, &abort_flag)) {
+        // the producer may have issued everything and left already: report here as well
+        if ((threadIdx.x & 31) == 0 && device_status) atomicOr(device_status, FASTAV_DEV_WAIT_EXPIRED);
+        return;
+      }
       const int key_base = key_begin + sl * kSlotKeys;
       const uint32_t slot = ring + stage * slot_bytes + lane_off;
       // The trip count is the same for every lane (the shuffles below need whole warps).
@@ -202,8 +208,9 @@ __global__ void __launch_bounds__(256) score_narrow_stats_kernel(Shapes s, const
   pdl_trigger();
   // the caller's arrays first: these loads overlap the predecessor's tail
   const int b = blockIdx.y, head = blockIdx.x / rq, r = blockIdx.x % rq;
-  const int row0 = cu_qlens[b], rows = min(cu_qlens[b + 1] - row0, rq);
-  const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
+  const Span seq = seq_span(s, cu_seqlens, b), qrows = row_span(s, cu_qlens, b);
+  const int row0 = qrows.first, rows = min(qrows.count, rq);
+  const int tok0 = seq.first, n = seq.count;
   pdl_wait();
   pdl_acquire(logits);
   if (r >= rows) return;
@@ -259,8 +266,9 @@ __global__ void __launch_bounds__(kFinalizeThreads) score_narrow_finalize_kernel
   pdl_trigger();
   // the caller's arrays first: these loads overlap the predecessor's tail
   const int b = blockIdx.y;
-  const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
-  const int row0 = cu_qlens[b], all_rows = cu_qlens[b + 1] - row0, rows = min(all_rows, rq);
+  const Span seq = seq_span(s, cu_seqlens, b), qrows = row_span(s, cu_qlens, b);
+  const int tok0 = seq.first, n = seq.count;
+  const int row0 = qrows.first, all_rows = qrows.count, rows = min(all_rows, rq);
   const int terms = s.hq * rows;
   pdl_wait();
   pdl_acquire(logits);

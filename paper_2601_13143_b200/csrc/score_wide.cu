@@ -200,8 +200,8 @@ static_assert(sizeof(Control) <= kCtrlBytes, "control block must fit its slot");
 // or one without scored rows).
 __device__ __forceinline__ int units_of_sequence(const Shapes& s, const int32_t* cu_seqlens, const int32_t* cu_qlens, int b,
                                                  int rows_per_chunk, int chunk_keys) {
-  const int n = cu_seqlens[b + 1] - cu_seqlens[b];
-  const int flat_rows = (cu_qlens[b + 1] - cu_qlens[b]) * s.group;
+  const int n = seq_span(s, cu_seqlens, b).count;
+  const int flat_rows = row_span(s, cu_qlens, b).count * s.group;
   if (n <= 0 || flat_rows <= 0) return 0;
   return s.hkv * ((flat_rows + rows_per_chunk - 1) / rows_per_chunk) * ((n + chunk_keys - 1) / chunk_keys);
 }
@@ -276,13 +276,18 @@ score_wide_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
     pdl_wait();
     return;
   }
+  // The host sized the key chunks so that a block's share fits its table; a longer share means the device's
+  // cu_seqlens describe more work than the host's total_tokens / batch did: the excess is left out and reported.
   const int n_mine = min(u1 - u0, kMaxUnits);
+  if (threadIdx.x == 0 && u1 - u0 > kMaxUnits && device_status) atomicOr(device_status, FASTAV_DEV_SHAPE_MISMATCH);
   // Unit `target` of the global order -> what to work on.  `b` is its sequence, `off` its index inside it.
   auto describe = [&](int b, int off, Unit& un) {
-    un.tok0 = cu_seqlens[b];
-    un.n = cu_seqlens[b + 1] - un.tok0;
-    un.row0 = cu_qlens[b];
-    const int flat_rows = (cu_qlens[b + 1] - un.row0) * s.group;
+    const Span seq = seq_span(s, cu_seqlens, b), rows = row_span(s, cu_qlens, b);
+    if ((seq.bad || rows.bad) && device_status) atomicOr(device_status, FASTAV_DEV_SHAPE_MISMATCH);
+    un.tok0 = seq.first;
+    un.n = seq.count;
+    un.row0 = rows.first;
+    const int flat_rows = rows.count * s.group;
     const int row_chunks = (flat_rows + rows_per_chunk - 1) / rows_per_chunk;
     const int key_chunks = (un.n + chunk_keys - 1) / chunk_keys;
     const int grc = off / key_chunks;
@@ -391,7 +396,10 @@ score_wide_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
   if (warp == 0) {
     // ---- TMA producer: one elected lane streams query tiles and K tiles ---------------------------
     if (lane == 0) {
-      if constexpr (SWEEP != 2) pdl_wait();  // first kernel of a chain: q and k may be what the previous kernel in the stream wrote
+      // q and k may be what the previous kernel in the stream wrote.  Sweep 2 is never the first kernel of a call,
+      // so it may fetch them ahead of its wait -- unless the call's first kernel was itself launched
+      // programmatically (FASTAV_CHAIN_CALLS): then the previous call's last kernel may still be running.
+      if (SWEEP != 2 || (s.flags & FASTAV_CHAIN_CALLS)) pdl_wait();
       int tile_no = 0, q_gen = 0;  // K tiles / query tiles issued so far
       bool ok = true;
       for (int u = 0; u < n_units && ok; ++u) {
@@ -688,7 +696,7 @@ __global__ void __launch_bounds__(256) score_wide_merge_kernel(Shapes s, const i
       const int mid = (lo + hi) >> 1;
       if (cu_qlens[mid] <= row) lo = mid; else hi = mid;
     }
-    const int n = cu_seqlens[lo + 1] - cu_seqlens[lo];
+    const int n = seq_span(s, cu_seqlens, lo).count;
     chunks = 2 * ((n + chunk_keys - 1) / chunk_keys);  // one entry per 64-key half of every tile run
   }
   pdl_wait();
@@ -722,8 +730,9 @@ __global__ void __launch_bounds__(kFinalizeThreads) score_wide_finalize_kernel(S
                                                                                float* __restrict__ scores) {
   pdl_trigger();
   const int b = blockIdx.y;
-  const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
-  const int rows = cu_qlens[b + 1] - cu_qlens[b];
+  const Span seq = seq_span(s, cu_seqlens, b);
+  const int tok0 = seq.first, n = seq.count;
+  const int rows = row_span(s, cu_qlens, b).count;
   const int row_chunks = (rows * s.group + rows_per_chunk - 1) / rows_per_chunk;
   const float inv = rows > 0 ? 1.0f / ((float)s.hq * (float)rows) : 0.f;
   pdl_wait();

@@ -1,4 +1,4 @@
-// Top-k keep set per sequence: "tokens with the lowest P% scores are removed" (Section 2.2).
+// Top-k keep set per sequence: the bottom-P % rule of Section 2.2 ("Fine pruning"), stated as "keep the k best".
 //
 // One thread block per sequence.  Scores become order-preserving 32-bit keys (protected tokens get
 // the largest key), held in shared memory when the sequence fits.  The k-th largest key T is found
@@ -80,7 +80,8 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
 
   pdl_trigger();
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
+  const Span seq = seq_span(s, cu_seqlens, b);  // never beyond what the key storage was sized for
+  const int tok0 = seq.first, n = seq.count;
   if (!kKeysInShared) keys = keys_global + tok0;
 
   const bool selecting = !kFromLogits || fl.do_select != 0;
@@ -89,15 +90,18 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
   __syncthreads();
   if (selecting) {
     int part = 0;
-    bool clamped = false;
+    bool clamped = false, mismatch = false;
     for (int i = tid; i <= b; i += kThreads) {
-      const int ni = cu_seqlens[i + 1] - cu_seqlens[i];
+      const Span si = seq_span(s, cu_seqlens, i);
+      const int ni = si.count;
+      mismatch |= si.bad;
       int ki = keep_counts[i];
       if (ki < 0 || ki > ni) { clamped = true; ki = ki < 0 ? 0 : ni; }
       if (i < b) part += ki;
     }
     if (part) atomicAdd(&sh.base, part);
     if (clamped && device_status) atomicOr(device_status, FASTAV_DEV_K_CLAMPED);
+    if (mismatch && device_status) atomicOr(device_status, FASTAV_DEV_SHAPE_MISMATCH);
   }
   int k = selecting ? keep_counts[b] : 0;
   k = k < 0 ? 0 : (k > n ? n : k);
@@ -110,7 +114,7 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
   if constexpr (kFromLogits) {
     pdl_acquire(fl.logits);
     float* lse_sh = reinterpret_cast<float*>(keys + (s.max_seqlen + s.max_seqlen / 32 + 1));
-    const int row0 = cu_qlens[b], all_rows = cu_qlens[b + 1] - row0, rows = min(all_rows, fl.rq);
+    const int all_rows = row_span(s, cu_qlens, b).count, rows = min(all_rows, fl.rq);
     const int terms = s.hq * rows;  // term i = (head i / rows, row i % rows)
     // where term i's logits start, in units of N floats: worked out once, not per token (no integer division in the loop below)
     int* term_row = reinterpret_cast<int*>(lse_sh + s.hq * fl.rq);
@@ -185,7 +189,8 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
   }
   __syncthreads();
   if (s.flags & FASTAV_PROTECT_QUERY_ROWS) {
-    for (int r = cu_qlens[b] + tid; r < cu_qlens[b + 1]; r += kThreads) {
+    const Span rows = checked_span(cu_qlens, b, s.total_q, s.total_q);
+    for (int r = rows.first + tid; r < rows.first + rows.count; r += kThreads) {
       const int j = q_idx[r];
       if (j >= 0 && j < n) keys[slot<kKeysInShared>(j)] = kProtectedKey;
     }
@@ -411,7 +416,8 @@ __global__ void __launch_bounds__(kThreads) select_topk_reg_kernel(Shapes s, con
 
   pdl_trigger();
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
+  const Span seq = seq_span(s, cu_seqlens, b);  // n <= max_seqlen <= kRegMaxKeys: every token has a register
+  const int tok0 = seq.first, n = seq.count;
   const bool by_rows = (s.flags & FASTAV_PROTECT_QUERY_ROWS) != 0;
   const int rounds = (n + kThreads - 1) / kThreads;  // <= kRegPer
 
@@ -422,21 +428,26 @@ __global__ void __launch_bounds__(kThreads) select_topk_reg_kernel(Shapes s, con
   __syncthreads();
   {
     int part = 0;
-    bool clamped = false;
+    bool clamped = false, mismatch = false;
     for (int i = tid; i <= b; i += kThreads) {
-      const int ni = cu_seqlens[i + 1] - cu_seqlens[i];
+      const Span si = seq_span(s, cu_seqlens, i);
+      const int ni = si.count;
+      mismatch |= si.bad;
       int ki = keep_counts[i];
       if (ki < 0 || ki > ni) { clamped = true; ki = ki < 0 ? 0 : ni; }
       if (i < b) part += ki;
     }
     if (part) atomicAdd(&sh.base, part);
     if (clamped && device_status) atomicOr(device_status, FASTAV_DEV_K_CLAMPED);
+    if (mismatch && device_status) atomicOr(device_status, FASTAV_DEV_SHAPE_MISMATCH);
   }
-  if (by_rows)
-    for (int r = cu_qlens[b] + tid; r < cu_qlens[b + 1]; r += kThreads) {
+  if (by_rows) {
+    const Span rows = checked_span(cu_qlens, b, s.total_q, s.total_q);
+    for (int r = rows.first + tid; r < rows.first + rows.count; r += kThreads) {
       const int j = q_idx[r];
       if (j >= 0 && j < n) atomicOr(&shared.row_bits[j >> 5], 1u << (j & 31));
     }
+  }
   int k = keep_counts[b];
   k = k < 0 ? 0 : (k > n ? n : k);
 
@@ -729,14 +740,15 @@ cudaError_t launch_narrow_tail(const Shapes& s, const float* logits, int rq, flo
 namespace {
 
 // counts[b] = number of kept tokens of sequence b.
-__global__ void __launch_bounds__(256) mask_count_kernel(int batch, const uint8_t* __restrict__ keep_mask,
+__global__ void __launch_bounds__(256) mask_count_kernel(Shapes s, const uint8_t* __restrict__ keep_mask,
                                                          const int32_t* __restrict__ cu_seqlens, int32_t* __restrict__ counts) {
   __shared__ int warp_sums[8];
   pdl_trigger();
   pdl_wait();
   pdl_acquire(keep_mask);
   const int b = blockIdx.x;
-  const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
+  const Span seq = checked_span(cu_seqlens, b, s.total_tokens, s.total_tokens);
+  const int tok0 = seq.first, n = seq.count;
   int c = 0;
   for (int j = threadIdx.x; j < n; j += 256) c += keep_mask[tok0 + j] != 0;
   c = __reduce_add_sync(0xFFFFFFFFu, c);
@@ -760,7 +772,9 @@ __global__ void __launch_bounds__(kThreads) mask_emit_kernel(Shapes s, const uin
   pdl_wait();
   pdl_acquire(counts);
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int tok0 = cu_seqlens[b], n = cu_seqlens[b + 1] - tok0;
+  const Span seq = checked_span(cu_seqlens, b, s.total_tokens, s.total_tokens);
+  const int tok0 = seq.first, n = seq.count;
+  if (tid == 0 && seq.bad && device_status) atomicOr(device_status, FASTAV_DEV_SHAPE_MISMATCH);
   if (tid == 0) base_sh = 0;
   __syncthreads();
   int part = 0;
@@ -814,7 +828,7 @@ extern "C" int32_t fastav_select_mask(const fastav_params* p, const uint8_t* kee
   s.flags = p->flags;
   int32_t* counts = static_cast<int32_t*>(workspace);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  cudaError_t e = launch_chained(mask_count_kernel, dim3(s.batch), dim3(256), 0, st, s.batch, keep_mask, cu_seqlens, counts);
+  cudaError_t e = launch_chained(mask_count_kernel, dim3(s.batch), dim3(256), 0, st, s, keep_mask, cu_seqlens, counts);
   if (e == cudaSuccess)
     e = launch_chained(mask_emit_kernel, dim3(s.batch), dim3(kThreads), 0, st, s, keep_mask, cu_seqlens, (const int32_t*)counts,
                        keep_idx_out, cu_keep_out, device_status);

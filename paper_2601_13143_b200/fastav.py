@@ -28,6 +28,8 @@ FASTAV_DEV_K_CLAMPED = 1
 FASTAV_DEV_PROTECT_OVERFLOW = 2
 FASTAV_DEV_WAIT_EXPIRED = 4
 FASTAV_DEV_BAD_INDEX = 8
+FASTAV_DEV_SHAPE_MISMATCH = 16
+FASTAV_DEV_SLOW_PATH = 32
 
 FASTAV_OK = 0
 FASTAV_ERR_INVALID_ARG = -1
@@ -104,12 +106,12 @@ def library() -> ctypes.CDLL:
         lib.fastav_compact.restype = ctypes.c_int32
         lib.fastav_compact.argtypes = [pp, i32p, i32p, i32p, vp, vp, i32p, i32p, vp, vp, vp, vp, i32p, vp]
         lib.fastav_prune.restype = ctypes.c_int32
-        lib.fastav_prune.argtypes = [pp, vp, i32p, i32p, vp, vp, i32p, i32p, vp, vp, i32p, vp, i32p, i32p, vp, i32p,
+        lib.fastav_prune.argtypes = [pp, vp, i32p, i32p, vp, vp, i32p, vp, i32p, vp, vp, i32p, vp, i32p, i32p, vp, i32p,
                                      vp, vp, vp, ctypes.c_size_t, i32p, vp]
         lib.fastav_host_arena_bytes.restype = ctypes.c_int32
         lib.fastav_host_arena_bytes.argtypes = [pp, ctypes.POINTER(ctypes.c_size_t)]
         lib.fastav_prune_host.restype = ctypes.c_int32
-        lib.fastav_prune_host.argtypes = [pp, vp, i32p, i32p, vp, vp, i32p, i32p, vp, vp, i32p, vp, i32p, i32p, vp, i32p,
+        lib.fastav_prune_host.argtypes = [pp, vp, i32p, i32p, vp, vp, i32p, vp, i32p, vp, vp, i32p, vp, i32p, i32p, vp, i32p,
                                           vp, vp, i32p, vp, ctypes.c_size_t, vp]
         lib.fastav_kernel_launches.restype = ctypes.c_int64
         lib.fastav_select_mask.restype = ctypes.c_int32
@@ -296,10 +298,10 @@ def fastav_compact(params, keep_idx, cu_keep, cu_seqlens, hidden_in=None, hidden
 
 def fastav_prune(params, q, q_idx, cu_qlens, k, v, cu_seqlens, keep_counts, protect_opt, hidden_in, pos_in, scores_out,
                  keep_idx_out, cu_keep_out, hidden_out, pos_out, k_out, v_out, workspace, device_status=None,
-                 stream=None) -> None:
+                 stream=None, lse_opt=None) -> None:
     ws, ws_bytes = _ws(workspace)
     _check(library().fastav_prune(ctypes.byref(params), _p(q), _p(q_idx), _p(cu_qlens), _p(k), _p(v), _p(cu_seqlens),
-                                  _p(keep_counts), _p(protect_opt), _p(hidden_in), _p(pos_in), _p(scores_out),
+                                  _p(lse_opt), _p(keep_counts), _p(protect_opt), _p(hidden_in), _p(pos_in), _p(scores_out),
                                   _p(keep_idx_out), _p(cu_keep_out), _p(hidden_out), _p(pos_out), _p(k_out), _p(v_out),
                                   ws, ws_bytes, _p(device_status), _stream(stream)), "fastav_prune")
 
@@ -316,14 +318,14 @@ def fastav_host_arena_bytes(params: fastav_params) -> int:
 
 def fastav_prune_host(params, q, q_idx, cu_qlens, k, v, cu_seqlens, keep_counts, protect_opt, hidden_in, pos_in, scores_out,
                       keep_idx_out, cu_keep_out, hidden_out, pos_out, k_out, v_out, status_out, device_arena,
-                      stream=None) -> None:
+                      stream=None, lse_opt=None) -> None:
     """All tensors are HOST tensors (pinned for asynchronous copies) except ``device_arena``."""
-    for t in (q, q_idx, cu_qlens, k, v, cu_seqlens, keep_counts, protect_opt, hidden_in, pos_in, scores_out, keep_idx_out,
+    for t in (q, q_idx, cu_qlens, k, v, cu_seqlens, lse_opt, keep_counts, protect_opt, hidden_in, pos_in, scores_out, keep_idx_out,
               cu_keep_out, hidden_out, pos_out, k_out, v_out, status_out):
         if t is not None and (t.is_cuda or not t.is_contiguous()):
             raise ValueError("fastav_prune_host takes contiguous host tensors")
     _check(library().fastav_prune_host(ctypes.byref(params), _p(q), _p(q_idx), _p(cu_qlens), _p(k), _p(v), _p(cu_seqlens),
-                                       _p(keep_counts), _p(protect_opt), _p(hidden_in), _p(pos_in), _p(scores_out),
+                                       _p(lse_opt), _p(keep_counts), _p(protect_opt), _p(hidden_in), _p(pos_in), _p(scores_out),
                                        _p(keep_idx_out), _p(cu_keep_out), _p(hidden_out), _p(pos_out), _p(k_out), _p(v_out),
                                        _p(status_out), _p(device_arena),
                                        ctypes.c_size_t(device_arena.numel() * device_arena.element_size()),
@@ -357,10 +359,10 @@ class PruneBuffers:
     workspace: torch.Tensor
     device_status: torch.Tensor
 
-    def prune(self, stream=None) -> None:
+    def prune(self, stream=None, lse_opt=None) -> None:
         fastav_prune(self.params, self.q, self.q_idx, self.cu_qlens, self.k, self.v, self.cu_seqlens, self.keep_counts,
                      self.protect, self.hidden, self.pos, self.scores, self.keep_idx, self.cu_keep, self.hidden_out,
-                     self.pos_out, self.k_out, self.v_out, self.workspace, self.device_status, stream)
+                     self.pos_out, self.k_out, self.v_out, self.workspace, self.device_status, stream, lse_opt=lse_opt)
 
     def score(self, stream=None) -> None:
         fastav_score(self.params, self.q, self.q_idx, self.cu_qlens, self.k, self.cu_seqlens, self.scores, self.workspace,

@@ -93,7 +93,7 @@ EXTRA_WORKLOADS = ("n3_fine_chain_13",)
 
 
 def keep_count(n: int, keep_ratio: float) -> int:
-    """Survivors when "the lowest P%" (P = 1 - keep_ratio) of n tokens are removed: the removed
+    """Survivors when the bottom P % by score (P = 1 - keep_ratio; Section 2.2, "Fine pruning") of n tokens are removed: the removed
     count is floor(P n)."""
     return n - int(math.floor((1.0 - keep_ratio) * n + 1e-6))
 
@@ -240,6 +240,12 @@ def make_stage(w: Workload, stage_index: int, lengths: list[int] | None = None, 
     return PruneInputs(model=m, q=q, k=k, v=v, hidden=hidden, pos=pos, cu_seqlens=cu, cu_qlens=cu_q, q_idx=q_idx,
                        keep_counts=keep_counts, modality=modality, anchors=anchors,
                        softmax_scale=1.0 / math.sqrt(m.head_dim), causal=True, protect_rows=True, layer=st.layer)
+
+
+def bf16_bits(t: torch.Tensor):
+    """bf16 tensor -> uint16 numpy view of the same bits (how inputs travel to a checker that takes bit patterns)."""
+    import numpy as np
+    return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
 
 
 def random_problem(seed: int, lens: list[int], rows: list[int], keeps: list[int], num_q_heads: int, num_kv_heads: int,

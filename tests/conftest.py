@@ -23,9 +23,7 @@ def pytest_collection_modifyitems(config, items):
             item.add_marker(skip)
 
 
-def bf16_bits(t: torch.Tensor) -> np.ndarray:
-    """bf16 tensor (CPU) -> uint16 numpy view of the same bits."""
-    return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+from paper_2601_13143_b200.workloads import bf16_bits  # noqa: E402  (bf16 tensor -> uint16 bit patterns)
 
 
 def to_bf16_bits(x) -> np.ndarray:

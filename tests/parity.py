@@ -140,6 +140,12 @@ def check_fused_against_oracle(p, buf: fastav.PruneBuffers, ref: dict, hidden=No
     total_keep = int(ref["cu_keep"][-1])
     gpu_keep = buf.keep_idx[:total_keep]
     differing = assert_keep_sets_match(p, gpu_keep, buf.cu_keep, ref["scores"], ref["keep_idx"], ref["cu_keep"], protect, what)
+    # Band or no band: the keep list must be THE top-k of the scores the GPU itself produced (integer work on
+    # fp32 bits, ties to the lower index), i.e. what the oracle's selector makes of those scores.
+    own_keep, own_cu = oracle.select(buf.scores.detach().cpu().numpy(), p.cu_seqlens.numpy(), p.keep_counts.numpy(),
+                                     None if protect is None else protect.numpy(), p.protect_rows, p.q_idx.numpy(), p.cu_qlens.numpy())
+    assert own_cu.tolist() == buf.cu_keep.cpu().tolist(), f"{what}: cu_keep differs from the selection on the GPU's own scores"
+    assert np.array_equal(gpu_keep.cpu().numpy(), own_keep), f"{what}: keep list is not the top-k of the GPU's own scores"
     mine = gather_rows(p, gpu_keep.cpu().numpy(), buf.cu_keep.cpu().numpy(), hidden, pos)
     assert_bits_equal(buf.hidden_out, mine["hidden"], what + " hidden (own keep set)")
     assert_bits_equal(buf.pos_out, mine["pos"], what + " pos (own keep set)")

@@ -800,3 +800,207 @@ def test_workspace_guard_band_and_equal_keys_tie_bit_exactly(lens, rows, hq, hkv
     bits = buf.scores.view(torch.int32).cpu()
     for a, b in twins:
         assert int(bits[a]) == int(bits[b]), (a, b)
+
+
+# ---- the fused call with the attention kernel's log-sum-exp -------------------------------------------
+
+@pytest.mark.parametrize("lens,rows,hq,hkv,d,hid", [
+    ([2048], [64], 28, 4, 128, 3584),                                   # the 2k global prune's shapes
+    ([4100, 1300], [128, 128], 32, 8, 128, 4096),                       # long-clip shapes, cut down to what the oracle does in seconds
+    ([1024, 3000, 1500, 2222, 1025], [32] * 5, 28, 4, 128, 3584),       # ragged serving batch shapes
+    ([900, 33], [1, 1], 8, 2, 64, 64),                                  # last-token query: the paper's fine stage
+])
+@pytest.mark.parametrize("host", [False, True])
+def test_fused_prune_with_the_attention_kernels_lse(lens, rows, hq, hkv, d, hid, host):
+    """fastav_prune / fastav_prune_host given lse_opt (float64 log-sum-exp rounded to fp32, as the layer's attention
+    kernel would return it): one sweep over K, same scores, keep set and survivor layout as the oracle."""
+    p = W.random_problem(seed=5, lens=lens, rows=rows, keeps=[n * 2 // 5 for n in lens], num_q_heads=hq, num_kv_heads=hkv,
+                         head_dim=d, hidden=hid)
+    p.protect_rows = True
+    lse = _natural_lse(p)
+    ref = parity.oracle_prune(p)
+    if not host:
+        buf = parity.to_device(p)
+        launches0 = fastav.fastav_kernel_launches()
+        buf.prune(lse_opt=lse.cuda())
+        with_lse = fastav.fastav_kernel_launches() - launches0
+        torch.cuda.synchronize()
+        stats = parity.check_fused_against_oracle(p, buf, ref, what=f"lse given, lens={lens}")
+        assert stats["device_status"] == 0
+        launches0 = fastav.fastav_kernel_launches()
+        buf.prune()
+        assert with_lse <= fastav.fastav_kernel_launches() - launches0     # never more kernels than the self-contained call
+        torch.cuda.synchronize()
+        parity.check_fused_against_oracle(p, buf, ref, what=f"self-contained, lens={lens}")
+        return
+    n, kk, rq = p.total_tokens, p.total_keep, int(p.cu_qlens[-1])
+    params = fastav.make_params(batch=len(lens), total_tokens=n, max_seqlen=max(lens), total_q=rq, max_qlen=max(rows), total_keep=kk,
+                                max_keep=int(p.keep_counts.max()), num_q_heads=hq, num_kv_heads=hkv, head_dim=d, hidden=hid,
+                                softmax_scale=p.softmax_scale, flags=parity.flags_of(p))
+    pin = lambda t: t.contiguous().pin_memory()
+    out = dict(scores=pin(torch.empty(n)), keep_idx=pin(torch.empty(kk, dtype=torch.int32)), cu_keep=pin(torch.empty(len(lens) + 1, dtype=torch.int32)),
+               hidden=pin(torch.empty(kk, hid, dtype=torch.bfloat16)), pos=pin(torch.empty(kk, dtype=torch.int32)),
+               k=pin(torch.empty(kk, hkv, d, dtype=torch.bfloat16)), v=pin(torch.empty(kk, hkv, d, dtype=torch.bfloat16)),
+               status=pin(torch.full((1,), -1, dtype=torch.int32)))
+    arena = torch.empty(fastav.fastav_host_arena_bytes(params), dtype=torch.uint8, device="cuda")
+    fastav.fastav_prune_host(params, pin(p.q), pin(p.q_idx), pin(p.cu_qlens), pin(p.k), pin(p.v), pin(p.cu_seqlens),
+                             pin(p.keep_counts), None, pin(p.hidden), pin(p.pos), out["scores"], out["keep_idx"], out["cu_keep"],
+                             out["hidden"], out["pos"], out["k"], out["v"], out["status"], arena, lse_opt=pin(lse))
+    torch.cuda.synchronize()
+    parity.assert_scores_close(out["scores"], ref["scores"], "host, lse given")
+    assert int(out["status"]) == 0 and out["cu_keep"].tolist() == ref["cu_keep"].tolist()
+    own_keep, _ = oracle.select(out["scores"].numpy(), p.cu_seqlens.numpy(), p.keep_counts.numpy(), None, True, p.q_idx.numpy(), p.cu_qlens.numpy())
+    assert np.array_equal(out["keep_idx"].numpy(), own_keep)
+    if np.array_equal(own_keep, ref["keep_idx"]):
+        for name in ("hidden", "pos", "k", "v"):
+            parity.assert_bits_equal(out[name], ref[name], "host " + name)
+
+
+def test_host_entry_point_refuses_before_it_copies_anything():
+    """A call the fused entry point would refuse must not have started its uploads: the arena keeps its contents."""
+    p = W.make_stage(W.WORKLOADS["c1_tiny"], 0)
+    m = p.model
+    n, kk = p.total_tokens, p.total_keep
+    params = fastav.make_params(batch=1, total_tokens=n, max_seqlen=n, total_q=4, max_qlen=4, total_keep=kk, max_keep=kk,
+                                num_q_heads=m.num_q_heads, num_kv_heads=m.num_kv_heads, head_dim=m.head_dim, hidden=m.hidden,
+                                softmax_scale=p.softmax_scale, flags=parity.flags_of(p) | fastav.FASTAV_SCORE_PATH_NARROW)
+    arena = torch.full((fastav.fastav_host_arena_bytes(params),), 0x3C, dtype=torch.uint8, device="cuda")
+    params.max_qlen = params.total_q = 64      # the forced matrix-vector path takes at most 4 scored rows: refused
+    pin = lambda t: t.contiguous().pin_memory()
+    q = pin(torch.zeros(64, m.num_q_heads, m.head_dim, dtype=torch.bfloat16))
+    q_idx = pin(torch.arange(64, dtype=torch.int32))
+    outs = [pin(torch.empty(n)), pin(torch.empty(kk, dtype=torch.int32)), pin(torch.empty(2, dtype=torch.int32)),
+            pin(torch.empty(kk, m.hidden, dtype=torch.bfloat16)), pin(torch.empty(kk, dtype=torch.int32)),
+            pin(torch.empty(kk, m.num_kv_heads, m.head_dim, dtype=torch.bfloat16)),
+            pin(torch.empty(kk, m.num_kv_heads, m.head_dim, dtype=torch.bfloat16)), pin(torch.zeros(1, dtype=torch.int32))]
+    big = torch.full((max(fastav.fastav_host_arena_bytes(params), arena.numel()),), 0x3C, dtype=torch.uint8, device="cuda")
+    with pytest.raises(fastav.FastavError) as err:
+        fastav.fastav_prune_host(params, q, q_idx, pin(torch.tensor([0, 64], dtype=torch.int32)), pin(p.k), pin(p.v), pin(p.cu_seqlens),
+                                 pin(p.keep_counts), None, pin(p.hidden), pin(p.pos), *outs, big)
+    assert err.value.status == fastav.FASTAV_ERR_UNSUPPORTED
+    torch.cuda.synchronize()
+    assert bool((big == 0x3C).all()), "copies were enqueued although the call was refused"
+
+
+# ---- chained calls whose tensors (not only index arrays) come from the call before -----------------------
+
+@pytest.mark.parametrize("lens,rows,hq,hkv,d", [([300, 200], [16, 8], 8, 2, 64), ([1500], [40], 4, 1, 128)])
+def test_chained_second_call_scores_the_keys_the_first_call_compacted(lens, rows, hq, hkv, d):
+    """Under FASTAV_CHAIN_CALLS only the INDEX arrays may be read early.  Here the second call's k and hidden are
+    the first call's k_out and hidden_out (a cache compacted in place of the layer's fresh projections), on shapes
+    whose tensor-core grids are far smaller than the GPU, so both calls' kernels can be resident together.  The
+    first call's outputs are poisoned before every repetition: keys fetched before the gather has finished would
+    be poison and change the second call's scores."""
+    keeps1 = [n // 2 for n in lens]
+    keeps2 = [k // 2 for k in keeps1]
+    p1 = W.random_problem(seed=31, lens=lens, rows=rows, keeps=keeps1, num_q_heads=hq, num_kv_heads=hkv, head_dim=d, hidden=128)
+    p1.protect_rows = True
+    ref1 = parity.oracle_prune(p1)
+    p2 = W.random_problem(seed=32, lens=keeps1, rows=rows, keeps=keeps2, num_q_heads=hq, num_kv_heads=hkv, head_dim=d, hidden=128)
+    p2.protect_rows = True
+    as_bf16 = lambda a: torch.from_numpy(a.view(np.int16).copy()).view(torch.bfloat16)
+    p2.k, p2.v = as_bf16(ref1["k"]), as_bf16(ref1["v"])      # what the first call must produce (checked below)
+    ref2 = parity.oracle_prune(p2, hidden=as_bf16(ref1["hidden"]), pos=torch.from_numpy(ref1["pos"]))
+    chain = fastav.FASTAV_CHAIN_CALLS | fastav.FASTAV_SCORE_PATH_WIDE
+    b1 = parity.to_device(p1, extra_flags=chain)
+    dev = lambda t: t.cuda()
+    b2 = fastav.make_buffers(q=dev(p2.q), q_idx=dev(p2.q_idx), cu_qlens=dev(p2.cu_qlens), k=b1.k_out, v=b1.v_out,
+                             cu_seqlens=dev(p2.cu_seqlens), keep_counts=dev(p2.keep_counts), hidden=b1.hidden_out, pos=b1.pos_out,
+                             softmax_scale=p2.softmax_scale, flags=parity.flags_of(p2) | chain, lens=keeps1, rows=rows, keeps=keeps2)
+    for rep in range(20):
+        for t in (b1.hidden_out, b1.k_out, b1.v_out):
+            t.view(torch.int16).fill_(0x7FC1)
+        b1.pos_out.fill_(-1)
+        b2.scores.fill_(float("nan"))
+        b1.prune()
+        b2.prune()
+        torch.cuda.synchronize()
+        s1 = parity.check_fused_against_oracle(p1, b1, ref1, what=f"first call, repetition {rep}")
+        assert s1["ambiguous_differing"] == 0
+        s2 = parity.check_fused_against_oracle(p2, b2, ref2, hidden=as_bf16(ref1["hidden"]), pos=torch.from_numpy(ref1["pos"]),
+                                               what=f"second call, repetition {rep}")
+        assert s2["device_status"] == 0
+
+
+# ---- the paper's fine chain replayed from one CUDA graph --------------------------------------------------
+
+def test_fine_chain_of_13_layers_replayed_from_one_graph_matches_the_oracle():
+    """Section 2.2 / 3.1: after the global stage the lowest 20 % go at each of the 13 later layers.  All 13 fused calls
+    are captured into ONE CUDA graph (stage s+1 reading stage s's hidden_out / pos_out in place), the graph is
+    replayed twice over poisoned outputs, and every stage of each replay is compared with the oracle chain."""
+    w = W.WORKLOADS["n3_fine_chain_13"]
+    stages, prev = [], None
+    for si in range(len(w.stages)):
+        p = W.make_stage(w, si)
+        lens = (p.cu_seqlens[1:] - p.cu_seqlens[:-1]).tolist()
+        rows = (p.cu_qlens[1:] - p.cu_qlens[:-1]).tolist()
+        buf = fastav.make_buffers(q=p.q.cuda(), q_idx=p.q_idx.cuda(), cu_qlens=p.cu_qlens.cuda(), k=p.k.cuda(), v=p.v.cuda(),
+                                  cu_seqlens=p.cu_seqlens.cuda(), keep_counts=p.keep_counts.cuda(),
+                                  hidden=p.hidden.cuda() if si == 0 else prev.hidden_out, pos=p.pos.cuda() if si == 0 else prev.pos_out,
+                                  softmax_scale=p.softmax_scale, flags=parity.flags_of(p) | fastav.FASTAV_CHAIN_CALLS, lens=lens, rows=rows,
+                                  keeps=p.keep_counts.tolist())
+        stages.append((p, buf))
+        prev = buf
+    refs, hidden, pos = [], stages[0][0].hidden, stages[0][0].pos
+    for p, _ in stages:
+        ref = parity.oracle_prune(p, hidden=hidden, pos=pos)
+        refs.append((ref, hidden, pos))
+        hidden = torch.from_numpy(ref["hidden"].view(np.int16).copy()).view(torch.bfloat16)
+        pos = torch.from_numpy(ref["pos"].copy())
+    for _, buf in stages:                       # one eager pass first: attribute set-up does not belong in a capture
+        buf.prune()
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        for _, buf in stages:
+            buf.prune(side)
+    for replay in range(2):
+        for _, buf in stages:
+            buf.scores.fill_(float("nan"))
+            buf.workspace.fill_(0xFF)
+            buf.keep_idx.fill_(-7)
+            buf.cu_keep.fill_(-7)
+            for t in (buf.hidden_out, buf.k_out, buf.v_out):
+                t.view(torch.int16).fill_(0x7FC1)
+            buf.pos_out.fill_(-1)
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        for si, ((p, buf), (ref, hidden, pos)) in enumerate(zip(stages, refs)):
+            stats = parity.check_fused_against_oracle(p, buf, ref, hidden=hidden, pos=pos, what=f"replay {replay}, stage {si}")
+            assert stats["device_status"] == 0
+            if stats["ambiguous_differing"]:    # a near-threshold token went the other way: later stages see another token set
+                break
+        else:
+            assert int(stages[-1][1].cu_keep[-1]) == stages[-1][0].total_keep
+
+
+# ---- host scalars that understate what the device arrays describe -----------------------------------------
+
+@pytest.mark.parametrize("true_len,claimed,entry", [(1500, 1000, "select"), (5000, 3000, "select"), (60_000, 52_000, "select"),
+                                                    (5000, 3000, "noalloc"), (1500, 1000, "prune_wide"), (1500, 1000, "prune_narrow")])
+def test_lengths_beyond_what_params_state_set_the_mismatch_bit(true_len, claimed, entry):
+    """Buffers are allocated for the TRUE lengths (so even an unguarded kernel would stay in bounds) while params
+    understates max_seqlen: the kernels size shared memory, registers and tables from the host scalars, so they
+    must cut the sequence down to what those promise and report FASTAV_DEV_SHAPE_MISMATCH."""
+    lens, keeps = [true_len, 200], [claimed // 2, 100]
+    rows = [1, 1] if entry == "prune_narrow" else [8, 8]
+    p = W.random_problem(seed=9, lens=lens, rows=rows, keeps=keeps, num_q_heads=4, num_kv_heads=2, head_dim=64, hidden=64)
+    p.protect_rows = True
+    buf = parity.to_device(p)
+    buf.params.max_seqlen = claimed
+    buf.scores.copy_(torch.rand(sum(lens)))
+    if entry == "select":
+        buf.select()
+    elif entry == "noalloc":
+        fastav.fastav_select_noalloc(buf.params, buf.scores, buf.cu_seqlens, buf.keep_counts, None, buf.q_idx, buf.cu_qlens,
+                                     buf.keep_idx, buf.cu_keep, buf.device_status)
+    else:
+        buf.prune()
+    torch.cuda.synchronize()
+    assert int(buf.device_status.cpu()) & fastav.FASTAV_DEV_SHAPE_MISMATCH
+    assert buf.cu_keep.cpu().tolist() == [0, keeps[0], keeps[0] + keeps[1]]
+    kept = buf.keep_idx.cpu().numpy()
+    assert kept[:keeps[0]].max() < claimed and (np.diff(kept[:keeps[0]]) > 0).all()

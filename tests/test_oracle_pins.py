@@ -293,6 +293,34 @@ def test_flops_column_of_table_4(golden_dir):
     assert oflops.removed_count(1024, 0.2) == 204 and oflops.removed_count(820, 0.2) == 164
 
 
+def test_reported_flops_agree_with_the_oracle_count_and_table_4(golden_dir):
+    """The benchmark's "prefill FLOPs removed" comes from the product's own restatement of the count; it must
+    give the oracle's relative figure (and hence Table 4's column) and the oracle's absolute saving."""
+    from paper_2601_13143_b200 import flops as pflops
+    from paper_2601_13143_b200 import workloads as W
+    with open(os.path.join(golden_dir, "table4_flops.json")) as f:
+        t = json.load(f)
+    a = t["assumed"]
+    for p_str, printed in t["printed"].items():
+        prunes = oflops.fastav_schedule(a["tokens"], t["num_layers"], t["global_layer"], a["global_keep"], int(p_str) / 100.0)
+        mine = pflops.schedule_flops(a["tokens"], prunes, t["num_layers"], a["hidden"], a["ffn"])
+        assert mine["relative"] == pytest.approx(oflops.relative_flops(a["tokens"], t["num_layers"], a["hidden"], a["ffn"], prunes), rel=1e-12)
+        assert abs(mine["relative"] - printed) <= t["tolerance_points"]
+        assert mine["removed"] == oflops.flops_removed(a["tokens"], t["num_layers"], a["hidden"], a["ffn"], prunes)
+    # the long audio-video workload's own schedule, per sequence
+    w = W.WORKLOADS["c4_long_av"]
+    lens = W.stage_lengths(w)
+    m = w.model
+    sched = {st.layer: lens[si + 1][0] for si, st in enumerate(w.stages)}
+    mine = pflops.schedule_flops(lens[0][0], sched, m.num_layers, m.hidden, m.ffn)
+    assert mine["relative"] == pytest.approx(oflops.relative_flops(lens[0][0], m.num_layers, m.hidden, m.ffn, sched), rel=1e-12)
+    assert mine["removed"] == oflops.flops_removed(lens[0][0], m.num_layers, m.hidden, m.ffn, sched)
+    # flops_removed itself, by hand: 3 layers of 10 tokens, D = 2, m = 3, prune to 4 tokens at layer 1:
+    # layer cost(n) = 4 n 4 + 2 n^2 2 + 2 n 6 = 28 n + 4 n^2 -> cost(10) = 680, cost(4) = 176; layers 2 and 3 save 504 each
+    assert oflops.flops_removed(10, 3, 2, 3, {1: 4}) == 1008
+    assert oflops.relative_flops(10, 3, 2, 3, {1: 4}) == pytest.approx(100.0 * (680 + 176 + 176) / (3 * 680))
+
+
 def test_mask_selection_equals_score_selection_on_indicator_scores():
     """A keep mask is the special case of the score rule in which kept tokens score 1, dropped ones 0 and
     k is the number of ones: the two oracle routes must agree (ties among the ones go to the lower index,

@@ -6,8 +6,9 @@ implicit synchronisation, a process whose memory pool was fully assigned at star
 library carries its own scratch (a fixed array of keys, one per token, 4 MiB) and this entry point
 uses it instead of a workspace.  The test calls it through the C ABI twice in a row on different
 inputs -- the second call finds the first call's keys still in the array -- and requires the same
-keep lists as ``fastav_select`` gives, bit for bit (integer work: no tolerance).  The file sorts
-last so that a run stopping at the first failure has already run every other test.
+keep lists as ``fastav_select`` gives, and as the CPU oracle's selector gives on the same scores, bit
+for bit (integer work: no tolerance).  The file sorts last so that a run stopping at the first failure
+has already run every other test.
 """
 import ctypes
 
@@ -15,6 +16,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2601_13143_b200 import fastav
 
 pytestmark = pytest.mark.gpu
@@ -32,7 +34,8 @@ def _problem(seed, lens, keeps, rows):
                                 total_keep=sum(keeps), max_keep=max(keeps), num_q_heads=4, num_kv_heads=2, head_dim=64,
                                 hidden=64, flags=fastav.FASTAV_PROTECT_QUERY_ROWS)
     dev = lambda a, dt: torch.as_tensor(a, dtype=dt).cuda()
-    return dict(params=params, scores=dev(scores, torch.float32), cu=dev(cu, torch.int32), keeps=dev(keeps, torch.int32),
+    host = dict(scores=scores, cu=cu, keeps=np.asarray(keeps, dtype=np.int32), protect=protect, q_idx=q_idx, cuq=cuq)
+    return dict(host=host, params=params, scores=dev(scores, torch.float32), cu=dev(cu, torch.int32), keeps=dev(keeps, torch.int32),
                 protect=dev(protect, torch.uint8), q_idx=dev(q_idx, torch.int32), cuq=dev(cuq, torch.int32),
                 total_keep=sum(keeps), batch=len(lens))
 
@@ -60,6 +63,11 @@ def test_select_noalloc_matches_select_on_two_calls_in_a_row():
         assert int(want_cu[-1]) == pr["total_keep"]
         assert torch.equal(got_idx, want_idx)                  # includes the untouched guard entries past the end
         assert int(got_status) == int(want_status)
+        # ... and both are what the plain definition gives (score descending, index ascending, protected first)
+        h = pr["host"]
+        ref_idx, ref_cu = oracle.select(h["scores"], h["cu"], h["keeps"], h["protect"], True, h["q_idx"], h["cuq"])
+        assert got_cu.cpu().tolist() == ref_cu.tolist()
+        assert np.array_equal(got_idx.cpu().numpy()[:pr["total_keep"]], ref_idx)
 
 
 def test_select_noalloc_rejects_sizes_beyond_its_scratch():
