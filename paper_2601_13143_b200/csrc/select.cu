@@ -15,6 +15,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "select_block.cuh"
 
 namespace fastav {
 namespace {
@@ -25,16 +26,6 @@ constexpr int kDigitBits = 13;  // long sequences; short ones (kShortKeys or few
 constexpr int kShortDigitBits = 11, kShortKeys = 2048;
 constexpr int kBins = 1 << kDigitBits;
 constexpr int kBinsPerThread = kBins / kThreads;  // bins one thread owns in the suffix scan, at most
-constexpr unsigned kProtectedKey = 0xFFFFFFFFu;
-constexpr int kDirectMax = 256;  // a bucket of at most this many keys is finished by counting ranks, not by more passes
-
-// fp32 -> uint32 with the same ordering as the float comparison (-0 and +0 compare equal).
-__device__ __forceinline__ unsigned order_key(float x) {
-  if (x == 0.0f) x = 0.0f;
-  const unsigned u = __float_as_uint(x);
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-
 struct SelectShared {
   unsigned hist[kBins];
   unsigned warp_a[kWarps], warp_b[kWarps];
@@ -383,304 +374,40 @@ __global__ void __launch_bounds__(kThreads) select_topk_kernel(Shapes s, const f
   }
 }
 
-// The same selection for sequences of kRegMinKeys < n <= kRegMaxKeys tokens with the keys in REGISTERS: thread t
-// holds tokens t, t + 1024, t + 2048, ... (coalesced loads, no shared-memory copy of the keys).  The block
-// sits on one SM, where every step that touches all keys is bound by the integer pipe: with the key in a
-// register a step costs a compare and a vote per key instead of a shared-memory read, its address and its
-// bounds arithmetic.  One histogram pass of 13-bit digits, then the direct finish on the chosen bin (further
-// passes only if that bin holds more than kDirectMax keys).  The stable scan goes by warp votes: kept keys per
-// (round, warp) cell, one scan over the at most 512 cells in index order, then each lane's rank inside its
-// cell; neighbouring lanes write neighbouring slots.
-constexpr int kRegPer = 16;
-constexpr int kRegMaxKeys = kThreads * kRegPer;
-constexpr int kRegMinKeys = kShortKeys;
-constexpr int kRegCells = kRegPer * kWarps;
+// Sequences of kBlockedMinKeys < n <= kBlockedMaxKeys tokens: one block per sequence with the BLOCKED layout (see
+// select_block.cuh) -- thread t owns PER consecutive tokens, the scores staged in shared memory and turned into
+// keys in place, the stable scan one prefix sum over the threads.
+constexpr int kBlockedMinKeys = kShortKeys;
+constexpr int kBlockedMaxKeys = kThreads * 32;
+using BlockedShared = SelectBlockedShared<kThreads, kDigitBits>;
 
-struct alignas(16) SelectRegShared {
-  SelectShared sel;
-  unsigned row_bits[kRegMaxKeys / 32];  // bit j: token j is a scored row that must survive
-  unsigned cell_gt[kRegCells], cell_eq[kRegCells];
-};
-
-__global__ void __launch_bounds__(kThreads) select_topk_reg_kernel(Shapes s, const float* __restrict__ scores,
-                                                                   const int32_t* __restrict__ cu_seqlens,
-                                                                   const int32_t* __restrict__ keep_counts,
-                                                                   const uint8_t* __restrict__ protect,
-                                                                   const int32_t* __restrict__ q_idx,
-                                                                   const int32_t* __restrict__ cu_qlens,
-                                                                   int32_t* __restrict__ keep_idx, int32_t* __restrict__ cu_keep,
-                                                                   int32_t* device_status) {
+template <int PER>
+__global__ void __launch_bounds__(kThreads) select_topk_blocked_kernel(Shapes s, const float* __restrict__ scores,
+                                                                       const int32_t* __restrict__ cu_seqlens,
+                                                                       const int32_t* __restrict__ keep_counts,
+                                                                       const uint8_t* __restrict__ protect,
+                                                                       const int32_t* __restrict__ q_idx,
+                                                                       const int32_t* __restrict__ cu_qlens,
+                                                                       int32_t* __restrict__ keep_idx, int32_t* __restrict__ cu_keep,
+                                                                       int32_t* device_status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  SelectRegShared& shared = *reinterpret_cast<SelectRegShared*>(smem_raw);
-  SelectShared& sh = shared.sel;
-
+  BlockedShared& shared = *reinterpret_cast<BlockedShared*>(smem_raw);
+  float* stage = reinterpret_cast<float*>(smem_raw + sizeof(BlockedShared));
   pdl_trigger();
-  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const Span seq = seq_span(s, cu_seqlens, b);  // n <= max_seqlen <= kRegMaxKeys: every token has a register
-  const int tok0 = seq.first, n = seq.count;
-  const bool by_rows = (s.flags & FASTAV_PROTECT_QUERY_ROWS) != 0;
-  const int rounds = (n + kThreads - 1) / kThreads;  // <= kRegPer
+  select_sequence_blocked<kThreads, PER, kDigitBits>(
+      shared, stage, s, blockIdx.x, threadIdx.x, scores, cu_seqlens, keep_counts, protect, q_idx, cu_qlens, keep_idx, cu_keep,
+      device_status, [] { __syncthreads(); }, [] { pdl_wait(); /* the scores are the previous kernel's output */ });
+}
 
-  if (tid == 0) { sh.base = 0; sh.protected_count = 0; sh.key_min = 0xFFFFFFFFu; sh.key_max = 0u; }
-  for (int i = tid; i < kBins; i += kThreads) sh.hist[i] = 0u;  // for the first pass
-  if (by_rows)
-    for (int i = tid; i < kRegMaxKeys / 32; i += kThreads) shared.row_bits[i] = 0u;
-  __syncthreads();
-  {
-    int part = 0;
-    bool clamped = false, mismatch = false;
-    for (int i = tid; i <= b; i += kThreads) {
-      const Span si = seq_span(s, cu_seqlens, i);
-      const int ni = si.count;
-      mismatch |= si.bad;
-      int ki = keep_counts[i];
-      if (ki < 0 || ki > ni) { clamped = true; ki = ki < 0 ? 0 : ni; }
-      if (i < b) part += ki;
-    }
-    if (part) atomicAdd(&sh.base, part);
-    if (clamped && device_status) atomicOr(device_status, FASTAV_DEV_K_CLAMPED);
-    if (mismatch && device_status) atomicOr(device_status, FASTAV_DEV_SHAPE_MISMATCH);
-  }
-  if (by_rows) {
-    const Span rows = checked_span(cu_qlens, b, s.total_q, s.total_q);
-    for (int r = rows.first + tid; r < rows.first + rows.count; r += kThreads) {
-      const int j = q_idx[r];
-      if (j >= 0 && j < n) atomicOr(&shared.row_bits[j >> 5], 1u << (j & 31));
-    }
-  }
-  int k = keep_counts[b];
-  k = k < 0 ? 0 : (k > n ? n : k);
-
-  pdl_wait();  // the scores are the previous kernel's output
-  pdl_acquire(scores);
-
-  float v[kRegPer];
-#pragma unroll
-  for (int u = 0; u < kRegPer; ++u) {
-    const int j = u * kThreads + tid;
-    v[u] = (u < rounds && j < n) ? chain_load(scores + tok0 + j) : 0.f;
-  }
-  unsigned prot = 0u;  // bit u: this thread's token of round u is protected
-  if (protect) {
-#pragma unroll
-    for (int u = 0; u < kRegPer; ++u) {
-      const int j = u * kThreads + tid;
-      if (u < rounds && j < n && protect[tok0 + j]) prot |= 1u << u;
-    }
-  }
-  __syncthreads();  // row_bits, sh.base complete
-  if (by_rows) {
-#pragma unroll
-    for (int u = 0; u < kRegPer; ++u)
-      if (u < rounds) prot |= ((shared.row_bits[u * kWarps + warp] >> lane) & 1u) << u;
-  }
-  // Keys.  A token that does not exist carries the protected key and is left out of every count by its index.
-  const bool lowest = (s.flags & FASTAV_SELECT_LOWEST) != 0;
-  unsigned key[kRegPer];
-  {
-    unsigned lo = 0xFFFFFFFFu, hi = 0u;
-    int n_prot = 0;
-#pragma unroll
-    for (int u = 0; u < kRegPer; ++u) {
-      key[u] = kProtectedKey;
-      if (u < rounds) {  // uniform
-        const bool exists = u * kThreads + tid < n;
-        unsigned x = order_key(lowest ? -v[u] : v[u]);
-        if (x == kProtectedKey) x = kProtectedKey - 1;  // only a NaN pattern lands here
-        if (!exists || ((prot >> u) & 1u)) x = kProtectedKey;
-        key[u] = x;
-        if (exists) {
-          if (x == kProtectedKey) ++n_prot;
-          else { lo = min(lo, x); hi = max(hi, x); }
-        }
-      }
-    }
-    lo = __reduce_min_sync(0xFFFFFFFFu, lo);
-    hi = __reduce_max_sync(0xFFFFFFFFu, hi);
-    n_prot = __reduce_add_sync(0xFFFFFFFFu, n_prot);
-    if (lane == 0) {
-      atomicMin(&sh.key_min, lo);
-      atomicMax(&sh.key_max, hi);
-      if (n_prot) atomicAdd(&sh.protected_count, n_prot);
-    }
-  }
-  __syncthreads();
-  const int base = sh.base, n_protected = sh.protected_count;
-  const unsigned key_min = sh.key_min, key_max = sh.key_max;
-  if (tid == 0) {
-    cu_keep[b + 1] = base + k;
-    if (b == 0) cu_keep[0] = 0;
-    if (n_protected > k && device_status) atomicOr(device_status, FASTAV_DEV_PROTECT_OVERFLOW);
-  }
-  if (k == 0 || n == 0) return;
-
-  unsigned T;
-  int need_eq;
-  if (k <= n_protected) {
-    T = kProtectedKey;
-    need_eq = k;
-  } else if (key_min == key_max) {
-    T = key_min;
-    need_eq = k - n_protected;
-  } else {
-    int bits_left = 32 - __clz(key_min ^ key_max);  // >= 1
-    if (tid == 0) {
-      sh.prefix = bits_left == 32 ? 0u : (key_min >> bits_left) << bits_left;
-      sh.remaining = k - n_protected;
-    }
-    __syncthreads();
-    for (int pass = 0; bits_left > 0; ++pass) {
-      const int width = min(kDigitBits, bits_left), shift = bits_left - width;
-      if (pass > 0) {  // the first pass finds the histogram zeroed by the prologue
-        for (int i = tid; i < kBins; i += kThreads) sh.hist[i] = 0u;
-        __syncthreads();
-      }
-      const unsigned prefix = sh.prefix;
-      const unsigned digit_mask = (1u << width) - 1u;
-      // the bits above this digit (none when bits_left is 32: the funnel shift clamps there and gives 0)
-      const unsigned above_want = __funnelshift_rc(prefix, 0u, bits_left);
-#pragma unroll
-      for (int u = 0; u < kRegPer; ++u) {
-        if (u < rounds) {  // uniform
-          const unsigned x = key[u];
-          // in the bucket: unprotected and equal to the prefix in the bits above this digit
-          const bool in_bucket = x != kProtectedKey && __funnelshift_rc(x, 0u, bits_left) == above_want;
-          const unsigned digit = in_bucket ? ((x >> shift) & digit_mask) : 0xFFFFu;
-          int same;
-          __match_all_sync(0xFFFFFFFFu, digit, &same);
-          if (same) {  // a run of equal scores (typically zeros): one add for the warp
-            if (in_bucket && lane == 0) atomicAdd(&sh.hist[digit], 32u);
-          } else if (in_bucket) {
-            atomicAdd(&sh.hist[digit], 1u);
-          }
-        }
-      }
-      __syncthreads();
-      // Suffix sums over the bins, kBinsPerThread consecutive bins per thread, to find the bin holding the wanted key.
-      unsigned h[kBinsPerThread];
-      unsigned own = 0;
-#pragma unroll
-      for (int i = 0; i < kBinsPerThread; i += 4) {
-        const uint4 q = *reinterpret_cast<const uint4*>(&sh.hist[kBinsPerThread * tid + i]);
-        h[i] = q.x; h[i + 1] = q.y; h[i + 2] = q.z; h[i + 3] = q.w;
-        own += q.x + q.y + q.z + q.w;
-      }
-      unsigned incl = own;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        const unsigned t = __shfl_down_sync(0xFFFFFFFFu, incl, d);
-        if (lane + d < 32) incl += t;
-      }
-      if (lane == 0) sh.warp_a[warp] = incl;
-      __syncthreads();
-      unsigned suffix = sh.warp_a[lane];
-      const unsigned own_total = suffix;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        const unsigned t = __shfl_down_sync(0xFFFFFFFFu, suffix, d);
-        if (lane + d < 32) suffix += t;
-      }
-      const unsigned above_warp = __shfl_sync(0xFFFFFFFFu, suffix - own_total, warp);
-      const unsigned above_me = above_warp + incl - own;
-      const unsigned rem = (unsigned)sh.remaining;
-      __syncthreads();  // everyone has read `remaining` (and warp_a) before the one owner rewrites it
-      if (above_me < rem && rem <= above_me + own) {
-        unsigned above = above_me;  // walk this thread's bins from the top
-#pragma unroll
-        for (int i = kBinsPerThread - 1; i >= 0; --i) {
-          if (above < rem && rem <= above + h[i]) {
-            sh.prefix = prefix | ((unsigned)(kBinsPerThread * tid + i) << shift);
-            sh.remaining = (int)(rem - above);
-            sh.bucket = (int)h[i];
-            sh.list_n = 0;
-          }
-          above += h[i];
-        }
-      }
-      __syncthreads();
-      bits_left = shift;
-      if (bits_left > 0 && sh.bucket <= kDirectMax) {
-        // Few keys left in the bucket: collect them and let each find its rank among them.
-        const unsigned want = sh.prefix >> bits_left;
-#pragma unroll
-        for (int u = 0; u < kRegPer; ++u)
-          if (u < rounds && key[u] != kProtectedKey && (key[u] >> bits_left) == want) sh.list[atomicAdd(&sh.list_n, 1)] = key[u];
-        __syncthreads();
-        const int count = sh.list_n, rem_in = sh.remaining;
-        __syncthreads();  // everyone has read `remaining` before an owner rewrites it
-        if (tid < count) {
-          const unsigned mine = sh.list[tid];
-          int above = 0, not_below = 0;
-          for (int i = 0; i < count; ++i) {
-            const unsigned other = sh.list[i];
-            above += other > mine;
-            not_below += other >= mine;
-          }
-          if (above < rem_in && rem_in <= not_below) {  // equal keys all write the same two values
-            sh.prefix = mine;
-            sh.remaining = rem_in - above;
-          }
-        }
-        __syncthreads();
-        bits_left = 0;
-      }
-    }
-    T = sh.prefix;
-    need_eq = sh.remaining;
-  }
-
-  // Stable compaction in index order.  Cell c = round * 32 + warp covers tokens 32 c .. 32 c + 31.
-  // A token that does not exist (it carries the protected key) is left out of both counts by its index.
-  const bool global_idx = (s.flags & FASTAV_KEEP_IDX_GLOBAL) != 0;
-#pragma unroll
-  for (int u = 0; u < kRegPer; ++u)
-    if (u < rounds) {
-      const bool exists = u * kThreads + tid < n;
-      const unsigned gt = __ballot_sync(0xFFFFFFFFu, exists && key[u] > T);
-      const unsigned eq = __ballot_sync(0xFFFFFFFFu, exists && key[u] == T);
-      if (lane == 0) { shared.cell_gt[u * kWarps + warp] = __popc(gt); shared.cell_eq[u * kWarps + warp] = __popc(eq); }
-    }
-  __syncthreads();
-  const int cells = rounds * kWarps;
-  unsigned cg_own = 0, ce_own = 0, cg_incl = 0, ce_incl = 0;
-  if (tid < kRegCells) {  // warps 0..15: exclusive scan of the cells, first inside each warp
-    cg_own = tid < cells ? shared.cell_gt[tid] : 0u;
-    ce_own = tid < cells ? shared.cell_eq[tid] : 0u;
-    cg_incl = cg_own; ce_incl = ce_own;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-      const unsigned a = __shfl_up_sync(0xFFFFFFFFu, cg_incl, d), c = __shfl_up_sync(0xFFFFFFFFu, ce_incl, d);
-      if (lane >= d) { cg_incl += a; ce_incl += c; }
-    }
-    if (lane == 31) { sh.warp_a[warp] = cg_incl; sh.warp_b[warp] = ce_incl; }
-  }
-  __syncthreads();
-  if (tid < kRegCells) {  // plus the totals of the warps before
-    unsigned pa = lane < kRegCells / 32 ? sh.warp_a[lane] : 0u, pb = lane < kRegCells / 32 ? sh.warp_b[lane] : 0u;
-    const unsigned ta = pa, tb = pb;
-#pragma unroll
-    for (int d = 1; d < kRegCells / 32; d <<= 1) {
-      const unsigned a = __shfl_up_sync(0xFFFFFFFFu, pa, d), c = __shfl_up_sync(0xFFFFFFFFu, pb, d);
-      if (lane >= d) { pa += a; pb += c; }
-    }
-    shared.cell_gt[tid] = cg_incl - cg_own + __shfl_sync(0xFFFFFFFFu, pa - ta, warp);
-    shared.cell_eq[tid] = ce_incl - ce_own + __shfl_sync(0xFFFFFFFFu, pb - tb, warp);
-  }
-  __syncthreads();
-  const unsigned below = (1u << lane) - 1u;
-#pragma unroll
-  for (int u = 0; u < kRegPer; ++u)
-    if (u < rounds) {
-      const int j = u * kThreads + tid;
-      const bool exists = j < n;
-      const bool is_gt = exists && key[u] > T, is_eq = exists && key[u] == T;
-      const unsigned gt = __ballot_sync(0xFFFFFFFFu, is_gt);
-      const unsigned eq = __ballot_sync(0xFFFFFFFFu, is_eq);
-      const int gt_before = (int)shared.cell_gt[u * kWarps + warp] + __popc(gt & below);
-      const int eq_before = (int)shared.cell_eq[u * kWarps + warp] + __popc(eq & below);
-      if (is_gt || (is_eq && eq_before < need_eq))
-        keep_idx[base + gt_before + min(eq_before, need_eq)] = global_idx ? tok0 + j : j;
-    }
+template <int PER>
+cudaError_t launch_blocked(const Shapes& s, const float* scores, const int32_t* cu_seqlens, const int32_t* keep_counts,
+                           const uint8_t* protect, const int32_t* q_idx, const int32_t* cu_qlens, int32_t* keep_idx, int32_t* cu_keep,
+                           int32_t* device_status, cudaStream_t stream) {
+  const size_t smem = sizeof(BlockedShared) + ((size_t)s.max_seqlen + s.max_seqlen / 32 + 1) * sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(select_topk_blocked_kernel<PER>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 1024);
+  if (e != cudaSuccess) return e;
+  return launch_chained(select_topk_blocked_kernel<PER>, dim3(s.batch), dim3(kThreads), smem, stream, s, scores, cu_seqlens,
+                        keep_counts, protect, q_idx, cu_qlens, keep_idx, cu_keep, device_status);
 }
 
 }  // namespace
@@ -693,11 +420,12 @@ cudaError_t launch_select(const Shapes& s, const Workspace& w, const float* scor
   const size_t want = fixed + ((size_t)s.max_seqlen + s.max_seqlen / 32 + 1) * sizeof(unsigned);
   constexpr size_t kMaxDynamic = 227 * 1024 - 1024;
   cudaError_t e;
-  if (s.max_seqlen > kRegMinKeys && s.max_seqlen <= kRegMaxKeys) {
-    e = cudaFuncSetAttribute(select_topk_reg_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SelectRegShared));
-    if (e != cudaSuccess) return e;
-    e = launch_chained(select_topk_reg_kernel, dim3(s.batch), dim3(kThreads), sizeof(SelectRegShared), stream, s, scores,
-                       cu_seqlens, keep_counts, protect, q_idx, cu_qlens, keep_idx, cu_keep, device_status);
+  if (s.max_seqlen > kBlockedMinKeys && s.max_seqlen <= kBlockedMaxKeys) {
+    // the fewest tokens per thread that cover the longest sequence: all 1024 threads share the work
+    if (s.max_seqlen <= kThreads * 4) e = launch_blocked<4>(s, scores, cu_seqlens, keep_counts, protect, q_idx, cu_qlens, keep_idx, cu_keep, device_status, stream);
+    else if (s.max_seqlen <= kThreads * 8) e = launch_blocked<8>(s, scores, cu_seqlens, keep_counts, protect, q_idx, cu_qlens, keep_idx, cu_keep, device_status, stream);
+    else if (s.max_seqlen <= kThreads * 16) e = launch_blocked<16>(s, scores, cu_seqlens, keep_counts, protect, q_idx, cu_qlens, keep_idx, cu_keep, device_status, stream);
+    else e = launch_blocked<32>(s, scores, cu_seqlens, keep_counts, protect, q_idx, cu_qlens, keep_idx, cu_keep, device_status, stream);
   } else if (want <= kMaxDynamic) {
     e = cudaFuncSetAttribute(select_topk_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynamic);
     if (e != cudaSuccess) return e;
