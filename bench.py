@@ -41,12 +41,36 @@ L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
 METRIC = "prune-step tokens/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# capture summarised under profiles/ (None until a capture of that kernel exists).
-NCU_TRAFFIC_BYTES = {
-    # profiles/compact_rows_bulk_c4_long_av.md and profiles/score_wide_c4_long_av.md (per launch; the score entry is sweep 1 + sweep 2)
-    "c4_long_av:0:compact": 590_784_256, "c4_long_av:1:compact": 396_079_360, "c4_long_av:0:score": 400_717_056,
-}
+
+
+def ncu_traffic_bytes() -> dict:
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch, as recorded in the ncu summaries under profiles/:
+    every line of the form ``traffic_bytes: <workload>:<stage>:<phase> = <bytes>`` there (none -> ``traffic`` is null)."""
+    out = {}
+    folder = os.path.join(ROOT, "profiles")
+    for name in sorted(os.listdir(folder)) if os.path.isdir(folder) else []:
+        if not name.endswith((".md", ".txt")):
+            continue
+        with open(os.path.join(folder, name)) as f:
+            for line in f:
+                if line.startswith("traffic_bytes:") and "=" in line:
+                    key, val = line[len("traffic_bytes:"):].split("=", 1)
+                    try:
+                        out[key.strip()] = int(val.strip().replace("_", "").replace(",", ""))
+                    except ValueError:
+                        pass
+    return out
+
+
+def cpu_model() -> str:
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
 
 
 def measured_peaks():
@@ -332,6 +356,98 @@ def rollout_line(device, peaks) -> dict:
             "device_status": int(status.cpu()), "launches_per_analysis": 2 + 3 * layers}
 
 
+def time_fused_chain(stages, stream, steps, warmup, flush_buf=None, lse=None) -> float:
+    """Mean ms per step of the fused chain (one fastav_prune per stage), CUDA events per step on `stream`.
+    ``lse[si]``: the attention kernel's log-sum-exp for stage si (None: the self-contained call)."""
+    def step():
+        for si, (_, buf) in enumerate(stages):
+            buf.prune(stream, lse_opt=None if lse is None else lse[si])
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    total = 0.0
+    for i in range(steps):
+        if flush_buf is not None:
+            flush_buf.fill_(i & 0xFF)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        step()
+        b.record(stream)
+        torch.cuda.synchronize()
+        total += a.elapsed_time(b)
+    return total / steps
+
+
+def graph_replay_ms(stages, stream, steps) -> float:
+    """The whole step (every stage's kernel chain) captured once and replayed: no host launch cost per step."""
+    side = torch.cuda.Stream()
+    side.wait_stream(stream)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        for _, buf in stages:
+            buf.prune(side)
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    ga, gb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ga.record()
+    for _ in range(steps):
+        graph.replay()
+    gb.record()
+    torch.cuda.synchronize()
+    return ga.elapsed_time(gb) / steps
+
+
+def other_workload_lines(device, stream, peaks, skip: str) -> list:
+    """The remaining configurations (and the paper's 13-layer fine chain), fused step only: ms per step, tokens/s and
+    the whole-step fraction of the HBM roofline.  Small ones flush L2 between steps; they are bound by launch
+    latency, not bandwidth, which is what the fractions show.  No CPU leg, a few seconds in all."""
+    out = []
+    for name in list(W.WORKLOAD_ORDER) + list(W.EXTRA_WORKLOADS):
+        if name == skip:
+            continue
+        w = W.WORKLOADS[name]
+        lens = W.stage_lengths(w)
+        stages = build_chain(w, device)
+        nbytes = [stage_bytes(p.model, p.total_tokens, int(p.cu_qlens[-1]), p.total_keep) for p, _ in stages]
+        flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=device) if nbytes[0]["total"] < 2 * L2_BYTES else None
+        ms = time_fused_chain(stages, stream, steps=10, warmup=3, flush_buf=flush)
+        total = sum(b["total"] for b in nbytes)
+        tokens = sum(sum(x) for x in lens[:-1])
+        line = {"workload": name, "stages": len(stages), "tokens_per_step": tokens, "ms_per_step": round(ms, 5),
+                "value": round(tokens / (ms * 1e-3), 1), "unit": "tokens/s", "algorithmic_bytes": total,
+                "step_hbm_frac_of_peak": round(total / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+                "l2": "flushed between steps" if flush is not None else "inputs larger than L2",
+                "device_status": sum(int(buf.device_status.cpu()) for _, buf in stages)}
+        if name in W.EXTRA_WORKLOADS or len(stages) > 2:
+            line["graph_replay_ms_per_step"] = round(graph_replay_ms(stages, stream, 10), 5)
+        out.append(line)
+        del stages, flush
+        torch.cuda.empty_cache()
+    return out
+
+
+def clock_check(fn, local, seconds=1.5) -> dict:
+    """Runs `fn` back to back for about `seconds` while nvidia-smi samples the SM clock: kernel time next to the
+    clock the SMs actually held under that load (the short timed region sees few samples)."""
+    torch.cuda.synchronize()
+    reps, t_end = 0, time.perf_counter() + seconds
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as cs:
+        a.record()
+        while time.perf_counter() < t_end:
+            for _ in range(50):
+                fn()
+            reps += 50
+            torch.cuda.synchronize()
+        b.record()
+        torch.cuda.synchronize()
+    summary = cs.summary()
+    ms = a.elapsed_time(b) / max(reps, 1)
+    return {"ms_back_to_back": round(ms, 5), "sm_mhz_median": summary["sm_mhz"], "samples": summary["samples"],
+            "reasons": summary["reasons"], "ms_times_ghz": None if not summary["sm_mhz"] else round(ms * summary["sm_mhz"] / 1e3, 5)}
+
+
 def workload_config(w: W.Workload, lens) -> dict:
     m = w.model
     return {"workload": w.name, "description": w.description, "batch": w.batch, "tokens_per_stage": [sum(x) for x in lens],
@@ -372,7 +488,8 @@ def main_reference(args, w, lens):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic", "config": workload_config(w, lens),
-        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": oracle.max_threads(), "kind": "oracle", "sample": desc},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": oracle.max_threads(), "kind": "oracle", "sample": desc,
+                         "cpu_model": cpu_model()},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 
@@ -387,6 +504,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-rollout", action="store_true", help="skip the secondary attention-rollout measurement")
+    ap.add_argument("--no-others", action="store_true", help="skip the fused-step lines of the other workloads")
+    ap.add_argument("--no-clock-check", action="store_true", help="skip the second-long loop of the dominant kernel (profiler runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -455,23 +574,7 @@ def main():
     barrier()
     graph_replay = None
     if args.graph:
-        # The whole step (every stage's kernel chain) captured once and replayed: no host launch cost per step.
-        side = torch.cuda.Stream()
-        side.wait_stream(stream)
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=side):
-            for _, buf in stages:
-                buf.prune(side)
-        for _ in range(3):
-            graph.replay()
-        torch.cuda.synchronize()
-        ga, gb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        ga.record()
-        for _ in range(args.steps):
-            graph.replay()
-        gb.record()
-        torch.cuda.synchronize()
-        graph_ms = R.max_over_ranks(ga.elapsed_time(gb) / args.steps, dist, device)
+        graph_ms = R.max_over_ranks(graph_replay_ms(stages, stream, args.steps), dist, device)
         graph_replay = {"ms_per_step": graph_ms, "value": R.aggregate_throughput(tokens_per_step, graph_ms, world), "unit": "tokens/s",
                         "note": "same kernels, enqueued by one graph launch; L2 not flushed between replays"}
     step_ms = [a.elapsed_time(b) for a, b in zip(starts, stops)]
@@ -498,6 +601,7 @@ def main():
 
     # ---- secondary line: the score when the caller hands over the attention kernel's log-sum-exp (one sweep) ----
     lse_ms = [None] * len(stages)
+    lse_all = [None] * len(stages)
     for si, (p, buf) in enumerate(stages):
         if int((p.cu_qlens[1:] - p.cu_qlens[:-1]).max()) <= 4:
             continue  # few scored rows: the statistics are a small part of that path
@@ -513,9 +617,17 @@ def main():
             torch.cuda.synchronize()
             if i >= 3:
                 lse_ms[si] = (lse_ms[si] or 0.0) + a.elapsed_time(b) / reps
-        del lse
+        lse_all[si] = lse
+
+    # ... and the whole fused step when the caller hands that log-sum-exp to fastav_prune (stages with few scored rows
+    # stay self-contained): the paper's method sits beside a FlashAttention-style kernel that has it already.
+    step_ms_lse = None
+    if any(x is not None for x in lse_all):
+        step_ms_lse = time_fused_chain(stages, stream, steps=reps, warmup=3, flush_buf=flush_buf, lse=lse_all)
+    del lse_all
 
     peaks = measured_peaks()
+    traffic_table = ncu_traffic_bytes()
     phases = []
     for si, ((p, _), b, t) in enumerate(zip(stages, bytes_per_stage, phase_ms)):
         rows_heads_tokens = sum(int(p.cu_qlens[i + 1] - p.cu_qlens[i]) * int(p.cu_seqlens[i + 1] - p.cu_seqlens[i])
@@ -530,7 +642,18 @@ def main():
     #   fraction of HBM peak and its MMAs of tensor peak, so it is reported as "alu": exponentials per second against
     #   the special-function-unit rate 148 SMs x 16 ex2/clk x SM clock (part of the exponentials run on the FMA pipe,
     #   so this is a reference rate rather than a hard ceiling).
-    clock_mhz = clocks.summary()["sm_mhz"] or peaks["sm_max_mhz"]
+    order = sorted(((si, name) for si in range(len(stages)) for name in ("score", "select", "compact")),
+                   key=lambda x: -phase_ms[x[0]][x[1]])
+    # the dominant kernel group back to back for a second or so, with the clock the SMs held meanwhile
+    top_si, top_name = order[0]
+    top_call = {"score": stages[top_si][1].score, "select": stages[top_si][1].select, "compact": stages[top_si][1].compact}[top_name]
+    clock = clock_check(lambda: top_call(stream), local) if rank == 0 and world == 1 and not args.no_clock_check else None
+    if clock is not None:
+        clock["kernel"] = f"{top_name} (stage {top_si})"
+
+    # The exponential rate is quoted against the clock the SMs HOLD under that kernel (sampled over a second or so of
+    # back-to-back launches when available: the timed region itself is too short for the power cap to bite).
+    clock_mhz = (clock or {}).get("sm_mhz_median") or clocks.summary()["sm_mhz"] or peaks["sm_max_mhz"]
     exp_peak = 148 * 16 * clock_mhz * 1e6 / 1e9  # Gexp/s
 
     def roofline_of(si, name):
@@ -540,16 +663,16 @@ def main():
             exps = 2 * phases[si]["score_exp2_per_sweep"]
             a = exps / (ms * 1e-3) / 1e9
             return {"kernel": f"score, tensor-core path (stage {si})", "bound": "alu", "achieved": round(a, 1), "peak": round(exp_peak, 1),
-                    "unit": "Gexp/s", "frac": round(a / exp_peak, 4), "of": f"derived: 148 SMs x 16 ex2/clk x {clock_mhz:.0f} MHz",
-                    "traffic": NCU_TRAFFIC_BYTES.get(f"{w.name}:{si}:{name}"), "exponentials": exps, "ms": round(ms, 5)}
+                    "unit": "Gexp/s", "frac": round(a / exp_peak, 4),
+                    "of": f"derived: 148 SMs x 16 ex2/clk x {clock_mhz:.0f} MHz (clock sampled under this kernel); at the maximum "
+                          f"clock {peaks['sm_max_mhz']:.0f} MHz the fraction is {a / (148 * 16 * peaks['sm_max_mhz'] * 1e-3):.4f}",
+                    "traffic": traffic_table.get(f"{w.name}:{si}:{name}"), "exponentials": exps, "ms": round(ms, 5)}
         b = bytes_per_stage[si][name]
         a = b / (ms * 1e-3) / 1e9
         return {"kernel": f"{name} (stage {si})", "bound": "hbm", "achieved": round(a, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": round(a / peaks["hbm_gbs"], 4), "of": peaks["source"], "traffic": NCU_TRAFFIC_BYTES.get(f"{w.name}:{si}:{name}"),
+                "frac": round(a / peaks["hbm_gbs"], 4), "of": peaks["source"], "traffic": traffic_table.get(f"{w.name}:{si}:{name}"),
                 "algorithmic_bytes": b, "ms": round(ms, 5)}
 
-    order = sorted(((si, name) for si in range(len(stages)) for name in ("score", "select", "compact")),
-                   key=lambda x: -phase_ms[x[0]][x[1]])
     roofline = roofline_of(*order[0])
     # the largest HBM-bound kernel as well, when the dominant one is not HBM-bound
     roofline_hbm = next(roofline_of(si, name) for si, name in order if roofline_of(si, name)["bound"] == "hbm")
@@ -598,10 +721,17 @@ def main():
             if dt >= 10.0 or dt * (passes + 1) / passes > 30.0:
                 break
         cpu = {"value": passes * stoks / dt, "unit": "tokens/s", "cores": oracle.max_threads(), "kind": "oracle", "seconds": round(dt, 3),
-               "sample": f"first sequence of each stage ({stoks} tokens) of {w.name}, {passes} passes"}
+               "sample": f"first sequence of each stage ({stoks} tokens) of {w.name}, {passes} passes", "cpu_model": cpu_model()}
+        # the same oracle on ONE thread (the plain parity reference), one pass over the same sample
+        t1 = time.perf_counter()
+        for x in sample:
+            oracle.prune(x["q"], x["k"], x["v"], x["hidden"], x["pos"], x["cu_seqlens"], x["cu_qlens"], x["q_idx"], x["keep_counts"],
+                         x["scale"], x["causal"], protect_rows=True, nthreads=1)
+        dt1 = time.perf_counter() - t1
+        cpu["single_thread"] = {"value": stoks / dt1, "unit": "tokens/s", "seconds": round(dt1, 3), "passes": 1}
 
     rollout = rollout_line(device, peaks) if rank == 0 and world == 1 and not args.no_rollout else None
-
+    others = other_workload_lines(device, stream, peaks, skip=w.name) if rank == 0 and world == 1 and not args.no_others else None
     if rank == 0:
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -612,8 +742,11 @@ def main():
             "step_hbm": {"algorithmic_bytes": bytes_per_step, "gbs": round(step_gbs, 1), "frac_of_peak": round(step_gbs / peaks["hbm_gbs"], 4),
                          "frac_of_nominal_8tbs": round(step_gbs / 8000.0, 4), "of": peaks["source"]},
             "roofline": roofline, "roofline_hbm": roofline_hbm, "compact_roofline": compact_rooflines, "phases": phases,
-            "prefill_flops": flops_removed(w, lens), "graph_replay": graph_replay, "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": launches,
-            "device_status": status, "clocks": clocks.summary(), "rollout": rollout}))
+            "prefill_flops": flops_removed(w, lens), "graph_replay": graph_replay,
+            "step_ms_given_attention_lse": None if step_ms_lse is None else round(step_ms_lse, 5),
+            "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": launches,
+            "device_status": status, "clocks": clocks.summary(), "dominant_kernel_clock_check": clock, "other_workloads": others,
+            "rollout": rollout}))
     if dist is not None:
         dist.destroy_process_group()
 
