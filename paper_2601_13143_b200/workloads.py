@@ -301,3 +301,11 @@ def positional_keep_mask(modality: torch.Tensor, cu_seqlens: torch.Tensor, keep_
             idx = torch.nonzero(seg == mod).flatten()
             mask[cu[b] + idx[m:]] = 0
     return mask
+
+
+def random_control_scores(seed: int, total_tokens: int) -> torch.Tensor:
+    """Scores of the "Random" control of the selector ablations (Tables 2-3): one seeded uniform draw per token,
+    fp32.  Handed to ``fastav_select`` in place of the attention scores, they make the keep set a seeded random
+    subset (protected tokens still survive, ties still go to the lower index).  Input construction only."""
+    gen = torch.Generator().manual_seed(seed)
+    return torch.rand(total_tokens, generator=gen, dtype=torch.float32)

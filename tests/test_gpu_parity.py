@@ -252,6 +252,28 @@ def test_select_lowest_keeps_the_least_attended_tokens():
     assert _select_case(lens, keeps, scores, protect, lowest=True) & ~fastav.FASTAV_DEV_PROTECT_OVERFLOW == 0
 
 
+def test_the_three_selectors_of_the_ablations_on_one_input():
+    """Tables 2-3 compare three ways of choosing what goes: the least attended tokens (the method), the most attended
+    ones, and a random subset.  The first two are fastav_select with and without FASTAV_SELECT_LOWEST on the attention
+    scores; the random control is fastav_select on one seeded uniform draw per token.  Each is checked against the
+    oracle's selection on the same scores, with the text rows protected."""
+    rng = np.random.default_rng(21)
+    lens, keeps = [2230, 744, 5000], [1115, 595, 1000]
+    n = sum(lens)
+    attention = rng.dirichlet(np.ones(64), size=(n + 63) // 64).reshape(-1)[:n].astype(np.float32)
+    random_scores = W.random_control_scores(seed=2601, total_tokens=n).numpy()
+    protect = np.zeros(n, dtype=np.uint8)
+    start = 0
+    for m in lens:  # the trailing text rows of every sequence survive whatever the selector
+        protect[start + m - 16:start + m] = 1
+        start += m
+    assert _select_case(lens, keeps, attention, protect) == 0
+    assert _select_case(lens, keeps, attention, protect, lowest=True) == 0
+    assert _select_case(lens, keeps, random_scores, protect) == 0
+    assert not np.array_equal(np.argsort(-random_scores[:lens[0]], kind="stable")[:keeps[0]],
+                              np.argsort(-attention[:lens[0]], kind="stable")[:keeps[0]])  # the control is a different subset
+
+
 def test_select_general_floats_negative_zero_and_inf():
     scores = np.array([0.0, -0.0, 1.5, -2.0, np.inf, 3e-39, -3e-39, 1.5, -np.inf, 0.0], dtype=np.float32)
     for k in range(0, 11):
