@@ -518,6 +518,30 @@ def test_compact_reports_out_of_range_indices():
 
 # ---- fused prune ------------------------------------------------------------------------------
 
+def test_prune_calls_on_two_streams_at_once_each_match_the_oracle():
+    """Two requests pruned at the same time on two streams, each with its own buffers and workspace (how a server
+    would run them): the calls share nothing, so each must give the oracle's result whatever the interleaving."""
+    shapes = [([3000, 517], [32, 8], [1200, 300], 8, 2, 128, 256), ([900, 2100, 33], [1, 1, 1], [700, 1500, 30], 28, 4, 128, 512)]
+    problems = [W.random_problem(seed=400 + i, lens=l, rows=r, keeps=k, num_q_heads=hq, num_kv_heads=hkv, head_dim=d, hidden=hid)
+                for i, (l, r, k, hq, hkv, d, hid) in enumerate(shapes)]
+    bufs = [parity.to_device(p) for p in problems]
+    refs = [parity.oracle_prune(p) for p in problems]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for buf in bufs:  # poison the outputs, so that a call that did not run cannot pass
+            buf.keep_idx.fill_(-3)
+            buf.scores.fill_(float("nan"))
+        torch.cuda.synchronize()
+        for _ in range(4):  # several calls deep on both streams, so that their kernels really interleave
+            for buf, st in zip(bufs, streams):
+                buf.prune(stream=st)
+        torch.cuda.synchronize()
+        for p, buf, ref in zip(problems, bufs, refs):
+            stats = parity.check_fused_against_oracle(p, buf, ref, what=f"two streams, repetition {rep}")
+            assert stats["device_status"] == 0
+
+
 @pytest.mark.parametrize("lens,rows,keeps,hq,hkv,d,hid", [
     ([9], [1], [4], 4, 2, 64, 64),
     ([129, 0, 64], [4, 0, 1], [64, 0, 64], 8, 2, 64, 128),
